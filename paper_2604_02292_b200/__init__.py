@@ -1,0 +1,18 @@
+"""HCCS (Head-Calibrated Clipped-Linear Softmax) inference kernels for NVIDIA B200.
+
+``workloads`` (numpy only) can be imported anywhere; everything else needs the
+compiled CUDA library ``csrc/libhccs.so`` and raises if it is missing.
+"""
+from . import workloads  # noqa: F401
+
+__all__ = ["workloads"]
+
+
+def __getattr__(name):
+    # the binding is loaded on first use so that the input generators work on hosts
+    # without the compiled library; a missing library is an ImportError, never a fallback
+    from . import binding
+    try:
+        return getattr(binding, name)
+    except AttributeError:
+        raise AttributeError(f"module {__name__!r} has no attribute {name!r}") from None

@@ -1,0 +1,59 @@
+"""Pins for the oracle's integer attention (Q.K^T -> requantise -> HCCS -> P.V)."""
+import math
+from fractions import Fraction
+
+import numpy as np
+
+from oracle import hccs_bigint as big
+from oracle import hccs_oracle as orc
+
+
+def test_requant_is_round_half_up_then_clamp():
+    """x = clamp(floor(acc*M / 2^sh + 1/2), -128, 127), checked with exact fractions."""
+    rng = np.random.default_rng(1)
+    cases = [(0, 1000, 20), (2 ** 18, 3840, 20), (-2 ** 18, 3840, 20), (1, 2 ** 19, 20),
+             (-1, 2 ** 19, 20), (3, 2 ** 19, 20), (-3, 2 ** 19, 20), (5, 1, 0), (-5, 3, 1)]
+    cases += [(int(a), int(m), 20) for a, m in zip(rng.integers(-2 ** 18, 2 ** 18, 400),
+                                                   rng.integers(768, 3841, 400))]
+    for acc, M, sh in cases:
+        exact = Fraction(acc * M, 2 ** sh) + Fraction(1, 2)
+        want = max(-128, min(127, math.floor(exact)))
+        assert orc.requant(acc, M, sh) == want, (acc, M, sh)
+    assert orc.requant(-1, 2 ** 19, 20) == 0        # -0.5 rounds up to 0
+    assert orc.requant(-3, 2 ** 19, 20) == -1       # -1.5 rounds up to -1
+    assert orc.requant(1, 2 ** 19, 20) == 1         # +0.5 rounds up to 1
+
+
+def test_attention_matches_matrix_route():
+    """The naive triple loops against the same composition done with library matrix
+    products (int64 matmul), vectorised requantisation and the pure-Python HCCS row."""
+    rng = np.random.default_rng(2)
+    Bt, H, L, d = 2, 3, 24, 8
+    Q = rng.integers(-64, 64, size=(Bt, H, L, d), dtype=np.int8)
+    K = rng.integers(-64, 64, size=(Bt, H, L, d), dtype=np.int8)
+    V = rng.integers(-64, 64, size=(Bt, H, L, d), dtype=np.int8)
+    M = np.array([90000, 170000, 400000], dtype=np.int32)     # spreads logits over int8
+    sh = 20
+    theta = np.array([(1300, 9, 100), (800, 30, 20), (1365, 127, 10)], dtype=np.int32)
+    for t in theta:
+        assert orc.check_params(*map(int, t), L) == 0
+    for mode in (0, orc.MODE_CLB, orc.MODE_CAUSAL):
+        O, lg, pr = orc.attention(Q, K, V, M, sh, theta, mode, want_intermediates=True)
+        acc = np.einsum("bhid,bhjd->bhij", Q.astype(np.int64), K.astype(np.int64))
+        x = np.clip((acc * M.astype(np.int64).reshape(1, H, 1, 1) + 2 ** (sh - 1)) >> sh, -128, 127)
+        assert (lg == x).all()
+        assert x.min() < -100 and x.max() > 100                # the clamp is exercised
+        P = np.zeros((Bt, H, L, L), dtype=np.int64)
+        for b, h, i in np.ndindex(Bt, H, L):
+            valid = [1 if j <= i else 0 for j in range(L)] if mode & orc.MODE_CAUSAL else None
+            P[b, h, i] = big.hccs_row(x[b, h, i].tolist(), theta[h], clb=bool(mode & orc.MODE_CLB),
+                                      valid=valid)
+        assert (pr == P).all()
+        want = P @ V.astype(np.int64)
+        assert (O == want).all()
+    # slices and row ranges only select independent work
+    O_all = orc.attention(Q, K, V, M, sh, theta, 0)
+    O_part = orc.attention(Q, K, V, M, sh, theta, 0, bh_range=(2, 5), q_range=(3, 11))
+    assert (O_part.reshape(-1, L, d)[2:5, 3:11] == O_all.reshape(-1, L, d)[2:5, 3:11]).all()
+    assert not O_part.reshape(-1, L, d)[:2].any() and not O_part.reshape(-1, L, d)[2:5, :3].any()
+    assert (orc.attention(Q, K, V, M, sh, theta, 0, threads=4) == O_all).all()
