@@ -3,15 +3,19 @@
 ``workloads`` (numpy only) can be imported anywhere; everything else needs the
 compiled CUDA library ``csrc/libhccs.so`` and raises if it is missing.
 """
+import importlib
+
 from . import workloads  # noqa: F401
 
 __all__ = ["workloads"]
 
 
 def __getattr__(name):
-    # the binding is loaded on first use so that the input generators work on hosts
-    # without the compiled library; a missing library is an ImportError, never a fallback
-    from . import binding
+    # The binding is loaded on first use so that the input generators work on hosts without
+    # the compiled library; a missing library is an ImportError, never a fallback.
+    if name.startswith("__"):
+        raise AttributeError(name)
+    binding = importlib.import_module(__name__ + ".binding")
     try:
         return getattr(binding, name)
     except AttributeError:

@@ -1,0 +1,62 @@
+// Internal declarations shared by the translation units of libhccs (not installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hccs.h"
+
+namespace hccs {
+
+// One head's theta in the form the kernels read with a single 16-byte load.
+struct __align__(16) HeadEntry {
+    int32_t B;        // B_h
+    int32_t S;        // S_h
+    uint32_t Drep;    // Dmax_h replicated into the four bytes of a word
+    int32_t D;        // Dmax_h
+};
+
+// Division of a 31-bit dividend by a runtime constant: q = (umulhi(n, mul) + n) >> shift.
+struct FastDiv {
+    uint32_t mul;
+    uint32_t shift;
+    uint32_t d;
+};
+FastDiv make_fastdiv(uint32_t d);
+
+// Everything a row kernel needs besides the two tensors.
+struct RowArgs {
+    const HeadEntry *table;   // device, num_heads entries
+    uint32_t *status;         // device status word (bounded waits report here)
+    int32_t rows;             // B*H*Lq
+    int32_t H, Lq, Lk;
+    int32_t causal_off;       // Lk - Lq
+    int32_t out_shift;        // OUT_SHIFT of Eq. 8
+    int32_t slice0;           // (b*H + h) index of flat row 0, mod H (views that start mid-tensor)
+    FastDiv div_Lq, div_H;
+};
+
+// Bits of the device status word.
+enum : uint32_t {
+    STATUS_ROW_TMA_TIMEOUT = 1u,     // CTA-per-row kernel: a bulk copy never completed
+    STATUS_FUSED_TIMEOUT = 2u,       // fused kernel: an mbarrier wait gave up
+};
+
+struct FusedArgs {
+    const int8_t *Q, *K, *V;
+    int32_t *O;
+    const HeadEntry *table;
+    const int32_t *requant_mult;   // device, H entries
+    uint32_t *status;
+    int32_t requant_shift;
+    int32_t B, H, L, d;
+    int32_t out_shift;
+    uint32_t flags;
+};
+
+// Launchers.  Each returns the CUDA error of the launch and adds to *launches.
+cudaError_t launch_rows(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                        cudaStream_t stream, uint64_t *launches);
+cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches);
+bool fused_shape_supported(int32_t L, int32_t d);
+
+}  // namespace hccs

@@ -1,0 +1,186 @@
+"""GPU parity: hccs_forward (through the C ABI) against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+
+from gpu_util import assert_same, forward_np, oracle_mode
+
+pytestmark = pytest.mark.gpu
+
+ALL_FLAGS = list(range(8))     # {u8,u16} x {div,clb} x {plain,causal}
+
+
+@pytest.fixture(scope="module")
+def ctx(hccs):
+    c = hccs.Context(0)
+    yield c
+    c.close()
+
+
+def _check(ctx, orc, wl, flags, out_shift=0, misalign=0, inplace=False, threads=8):
+    ctx.hccs_params_upload(wl.theta, wl.n_design, out_shift)
+    got = forward_np(ctx, wl.logits, flags, misalign=misalign, inplace=inplace)
+    want = orc.forward(wl.logits, wl.theta, oracle_mode(orc, flags), out_shift, threads=threads)
+    assert_same(got, want, f"{wl.name} shape={wl.shape} flags={flags} os={out_shift} mis={misalign}")
+    assert ctx.hccs_device_status() == 0
+
+
+@pytest.mark.parametrize("flags", ALL_FLAGS)
+def test_config1_all_modes(ctx, oracle, hccs, flags):
+    wl = hccs.workloads.make_config(1)
+    _check(ctx, oracle, wl, flags)
+
+
+@pytest.mark.parametrize("c,batch", [(2, 33), (3, 5), (4, 2)])
+@pytest.mark.parametrize("flags", ALL_FLAGS)
+def test_reduced_configs_all_modes(ctx, oracle, hccs, c, batch, flags):
+    wl = hccs.workloads.make_config(c, batch=batch)
+    _check(ctx, oracle, wl, flags)
+
+
+# row lengths around every dispatch boundary: lane-group sizes, two vectors per lane, the
+# CTA-per-row kernel, ragged tails and lengths that are no multiple of 16
+LENGTHS = [1, 2, 3, 15, 16, 17, 31, 32, 33, 48, 64, 80, 96, 100, 112, 128, 144, 256, 257, 272, 384,
+           496, 512, 528, 1000, 1008, 1024, 1040, 2048, 2064, 4096, 5000, 8192]
+
+
+@pytest.mark.parametrize("Lk", LENGTHS)
+def test_row_lengths(ctx, oracle, hccs, Lk):
+    for kind, flags, shape in (("gauss", 0, (2, 3, 7, Lk)), ("uniform", 1, (1, 5, 4, Lk)),
+                               ("laplace", 2, (3, 2, 5, Lk)), ("extreme", 3, (1, 1, 9, Lk)),
+                               ("const", 0, (1, 2, 3, Lk))):
+        wl = hccs.workloads.make_rows(1000 + Lk, shape, kind=kind)
+        _check(ctx, oracle, wl, flags)
+
+
+@pytest.mark.parametrize("Lq,Lk", [(1, 64), (5, 64), (64, 5), (100, 128), (128, 100), (33, 512),
+                                   (40, 1024), (7, 2048), (3, 1), (130, 144), (2100, 2048)])
+def test_causal_alignment(ctx, oracle, hccs, Lq, Lk):
+    for flags in (4, 5, 6, 7):
+        wl = hccs.workloads.make_rows(50 + Lq + Lk, (2, 3, Lq, Lk), kind="gauss")
+        _check(ctx, oracle, wl, flags)
+
+
+def test_shorter_rows_than_designed(ctx, oracle, hccs):
+    for Lk in (16, 48, 64, 100):
+        wl = hccs.workloads.make_rows(7, (2, 4, 9, Lk), n_design=128, kind="gauss")
+        for flags in (0, 1, 2, 3, 4):
+            _check(ctx, oracle, wl, flags)
+
+
+@pytest.mark.parametrize("out_shift", [0, 1, 2, 5])
+def test_out_shift(ctx, oracle, hccs, out_shift):
+    for Lk in (64, 100, 2048):
+        wl = hccs.workloads.make_rows(3, (2, 3, 8, Lk), kind="gauss")
+        for flags in (0, 2, 4):
+            _check(ctx, oracle, wl, flags, out_shift=out_shift)
+
+
+@pytest.mark.parametrize("misalign", [1, 4, 8, 15])
+def test_unaligned_pointers(ctx, oracle, hccs, misalign):
+    for Lk in (64, 128, 2048):
+        wl = hccs.workloads.make_rows(9, (1, 2, 6, Lk), kind="gauss")
+        for flags in (0, 1):
+            _check(ctx, oracle, wl, flags, misalign=misalign)
+
+
+def test_in_place(ctx, oracle, hccs):
+    for Lk in (64, 100, 512, 1024, 4096):
+        wl = hccs.workloads.make_rows(21, (2, 2, 10, Lk), kind="gauss")
+        for flags in (0, 2, 4):
+            _check(ctx, oracle, wl, flags, inplace=True)
+
+
+def test_many_heads_and_odd_head_count(ctx, oracle, hccs):
+    wl = hccs.workloads.make_rows(5, (3, 67, 3, 64), kind="gauss")
+    _check(ctx, oracle, wl, 0)
+    wl = hccs.workloads.make_rows(6, (2, 200, 2, 32), kind="laplace")
+    _check(ctx, oracle, wl, 1)
+
+
+def test_every_row_sum_is_reached(ctx, oracle, hccs):
+    """Rows built so that Z takes every value in 1..32767 (the exact divide per row is the one
+    scalar step): Lk = 16 with a table designed for 256 keys lets B start at 1."""
+    rows, thetas = [], []
+    # Z = nv*B - S*sum(delta): one key (nv = 1 through the causal mask) gives Z = B = 1..127
+    # 16 keys, S = 1: Z = 16*B - sum(delta), sum(delta) in 0..15*min(D, 255)
+    H = 127
+    x = np.zeros((1, H, 16, 16), dtype=np.int8)
+    theta = np.zeros((H, 3), dtype=np.int32)
+    rng = np.random.default_rng(1)
+    for h in range(H):
+        B = h + 1                       # n_design = 256: 1 <= B <= 127, floor score 1
+        D = max(1, min(127, B - 1))
+        theta[h] = (B, 1 if B - D >= 1 else 0, D)
+        x[0, h] = rng.integers(-128, 128, size=(16, 16))
+    wl = hccs.workloads.Workload("allZ-small", x.shape, 4, 256, theta, logits=x)
+    _check(ctx, oracle, wl, 4)
+    _check(ctx, oracle, wl, 5)
+    # large Z: Lk = 16, n_design = 16 -> B up to 2047; sweep sum(delta) through the row contents
+    H = 256
+    theta = np.zeros((H, 3), dtype=np.int32)
+    Bs = np.linspace(143, 2047, H).astype(np.int32)
+    theta[:, 0], theta[:, 1], theta[:, 2] = Bs, 1, 127
+    x = np.full((8, H, 16, 16), -128, dtype=np.int8)
+    x[..., 0] = 127                                     # the max; the others sit up to 255 below
+    steps = rng.integers(0, 128, size=(8, H, 16, 15))
+    x[..., 1:] = (127 - steps).astype(np.int8)
+    wl = hccs.workloads.Workload("allZ-large", x.shape, 0, 16, theta, logits=x)
+    seen = set()
+    for flags in (0, 1):
+        _check(ctx, oracle, wl, flags)
+    for b, h, i in np.ndindex(8, H, 16):
+        seen.add(int(16 * Bs[h] - np.minimum(127 - x[b, h, i].astype(int), 127).sum()))
+    assert len(seen) > 10000
+
+
+def test_empty_tensors_and_errors(ctx, hccs):
+    import torch
+    ctx.hccs_params_upload([(300, 3, 85)] * 4, 64)
+    dev = torch.device("cuda", 0)
+    e = torch.empty((0, 4, 64, 64), dtype=torch.int8, device=dev)
+    ctx.hccs_forward(e, e.view(torch.uint8), 0)                       # no rows: OK, no launch
+    e = torch.empty((2, 4, 0, 64), dtype=torch.int8, device=dev)
+    ctx.hccs_forward(e, e.view(torch.uint8), 0)
+    x = torch.zeros((1, 4, 8, 64), dtype=torch.int8, device=dev)
+    p = torch.zeros((1, 4, 8, 64), dtype=torch.uint8, device=dev)
+    n0 = ctx.hccs_launch_count()
+    ctx.hccs_forward(x, p, 0)
+    assert ctx.hccs_launch_count() == n0 + 1
+    with pytest.raises(hccs.HccsError) as ei:                         # wrong head count
+        ctx.hccs_forward(torch.zeros((1, 3, 8, 64), dtype=torch.int8, device=dev),
+                         torch.zeros((1, 3, 8, 64), dtype=torch.uint8, device=dev), 0)
+    assert ei.value.status == hccs.HCCS_ERR_INVALID_ARG
+    with pytest.raises(hccs.HccsError) as ei:                         # longer than designed
+        ctx.hccs_forward(torch.zeros((1, 4, 8, 80), dtype=torch.int8, device=dev),
+                         torch.zeros((1, 4, 8, 80), dtype=torch.uint8, device=dev), 0)
+    assert ei.value.status == hccs.HCCS_ERR_CONSTRAINT
+    with pytest.raises(hccs.HccsError) as ei:                         # unknown flag
+        ctx.hccs_forward(x, p, 8)
+    assert ei.value.status == hccs.HCCS_ERR_INVALID_ARG
+    with pytest.raises(hccs.HccsError) as ei:                         # constraint violation
+        ctx.hccs_params_upload([(300, 3, 85), (200, 3, 85)], 64)
+    assert ei.value.status == hccs.HCCS_ERR_CONSTRAINT and "head 1" in str(ei.value)
+    ctx.hccs_forward(x, p, 0)                                         # the old table is still in force
+    fresh = hccs.Context(0)
+    with pytest.raises(hccs.HccsError) as ei:
+        fresh.hccs_forward(x, p, 0)
+    assert ei.value.status == hccs.HCCS_ERR_NOT_UPLOADED
+    fresh.close()
+    assert ctx.hccs_launch_count() == n0 + 2
+
+
+def test_forward_host_matches_forward(ctx, oracle, hccs):
+    import torch
+    for c, batch, flags in ((2, 40, 0), (3, 6, 4), (4, 3, 1), (2, 700, 0)):
+        wl = hccs.workloads.make_config(c, batch=batch)
+        ctx.hccs_params_upload(wl.theta, wl.n_design)
+        f = flags | wl.flags
+        xin = torch.from_numpy(wl.logits).pin_memory()
+        odt = torch.uint16 if f & 1 else torch.uint8
+        out = torch.empty(wl.logits.shape, dtype=odt).pin_memory()
+        s_in = torch.empty(wl.logits.shape, dtype=torch.int8, device="cuda")
+        s_out = torch.empty(wl.logits.shape, dtype=odt, device="cuda")
+        ctx.hccs_forward_host(xin, out, s_in, s_out, f)
+        torch.cuda.synchronize()
+        want = oracle.forward(wl.logits, wl.theta, oracle_mode(oracle, f), threads=8)
+        assert_same(out.numpy(), want, f"forward_host config{c}")
