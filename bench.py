@@ -200,7 +200,8 @@ def run_ours(args):
         ctx.hccs_forward(xs[s % nbuf], ps[s % nbuf], flags, stream=sptr)
     barrier()
     sampler = ClockSampler(local)
-    if rank == 0:
+    full = not args.kernel_only
+    if rank == 0 and full:
         sampler.start()
         time.sleep(0.3)
     launches0 = ctx.hccs_launch_count()
@@ -218,20 +219,20 @@ def run_ours(args):
         best_ms = float(t.item())
     launches = ctx.hccs_launch_count() - launches0
     # keep the GPU busy long enough for the clock sampler to see it under load
-    if rank == 0:
+    if rank == 0 and full:
         t_end = time.time() + 1.0
         while time.time() < t_end:
             for s in range(64):
                 ctx.hccs_forward(xs[s % nbuf], ps[s % nbuf], flags, stream=sptr)
             torch.cuda.synchronize()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop() if rank == 0 and full else None
     ms_per_step = best_ms / args.steps
     rows_per_s = world * wl.rows / (ms_per_step * 1e-3)
 
     # ---------------- end to end: host tensors in, host tensors out, through hccs_forward_host
     host_p = torch.empty(wl.logits.shape, dtype=torch.uint8).pin_memory()
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
+    e2e_steps = max(3, min(args.steps, 10)) if full else 0
+    for _ in range(2 if full else 0):
         ctx.hccs_forward_host(host_x, host_p, xs[0], ps[0], flags, stream=sptr)
     barrier()
     e0.record(stream)
@@ -244,7 +245,7 @@ def run_ours(args):
         t = torch.tensor([e2e_ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
-    e2e_rows_per_s = world * wl.rows * e2e_steps / (e2e_ms * 1e-3)
+    e2e_rows_per_s = world * wl.rows * e2e_steps / (e2e_ms * 1e-3) if full else None
     status = ctx.hccs_device_status()
 
     if rank == 0:
@@ -259,9 +260,10 @@ def run_ours(args):
         nb = max(1, wl.shape[0] // 64)
         want = orc.forward(wl.logits[:nb], wl.theta, mode, threads=os.cpu_count() or 1)
         mism = int((ps[0][:nb].cpu().numpy() != want).sum())
-        mism += int((host_p[:nb].numpy() != want).sum())
+        if full:
+            mism += int((host_p[:nb].numpy() != want).sum())
         cpu_cores = os.cpu_count() or 1
-        cpu_rate, cpu_passes, cpu_dt = cpu_oracle_rate(wl, 2.5, cpu_cores) if world == 1 else (None, 0, 0)
+        cpu_rate, cpu_passes, cpu_dt = cpu_oracle_rate(wl, 2.5, cpu_cores) if world == 1 and full else (None, 0, 0)
         line = {
             "metric": METRIC, "value": rows_per_s, "unit": "rows/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
@@ -279,8 +281,8 @@ def run_ours(args):
                          "true_bytes_per_launch": true_bytes,
                          "achieved_true_bytes": true_bytes / kernel_s / 1e9},
             "e2e": {"value": e2e_rows_per_s, "unit": "rows/s", "h2d_bytes_per_step": nbytes,
-                    "d2h_bytes_per_step": nbytes, "ms_per_step": e2e_ms / e2e_steps,
-                    "steps": e2e_steps},
+                    "d2h_bytes_per_step": nbytes,
+                    "ms_per_step": e2e_ms / e2e_steps if full else None, "steps": e2e_steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
             "parity_mismatches": mism,
@@ -304,6 +306,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only the device-resident timing (for profiler captures): no end-to-end leg, "
+                         "no CPU baseline, no clock sampling")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

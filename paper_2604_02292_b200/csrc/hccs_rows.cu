@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(256) rows_lanegroup_kernel(const int8_t *__res
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int col = (sub + v * G) * 16;
-            int c = live && col < a.Lk ? min(nv[u] - col, 16) : -1;
+            int c = live && col < a.Lk ? max(min(nv[u] - col, 16), 0) : -1;
             cnt[u][v] = c;                                   // -1: nothing to write either
             w[u][v] = make_uint4(0, 0, 0, 0);
             if (c > 0)
