@@ -1,0 +1,56 @@
+// Device helpers shared by the row kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hccs_internal.h"
+
+namespace hccs {
+
+constexpr uint32_t kTprimeU8 = 255u << 15;   // 255 * 2^R, R = INV_SHIFT = 15 (Eq. 8)
+constexpr uint32_t kTprimeU16 = 32767u;      // T for int16 output (Eq. 6)
+
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv &f) {
+    return (__umulhi(n, f.mul) + n) >> f.shift;
+}
+
+// (head, query index) of flat row r: head = ((r / Lq) + slice0) mod H, i = r mod Lq.
+__device__ __forceinline__ void row_coords(uint32_t r, const RowArgs &a, uint32_t &head, uint32_t &i) {
+    uint32_t bh = fast_div(r, a.div_Lq);
+    i = r - bh * (uint32_t)a.Lq;
+    bh += (uint32_t)a.slice0;
+    uint32_t b = fast_div(bh, a.div_H);
+    head = bh - b * (uint32_t)a.H;
+}
+
+// Stage 5 of the kernel overview: the one scalar operation per row, rho = floor(T'/Z) (Eq. 6,
+// Eq. 8) or T' >> floor(log2 Z) (Eq. 9).  Z >= 1.
+//
+// The exact quotient is taken without an integer divide: a float estimate that is never above
+// T'/Z and less than one below it, then one upward correction.  rcp.approx and the
+// round-toward-zero multiply are each within 2^-22 relative; the numerator is pre-scaled by
+// (1 - 2^-20), so the estimate lies in (T'/Z * (1 - 2^-19.5) - 1, T'/Z]; for quotients up to
+// 2^15 the relative part is below 0.05, hence floor(estimate) is q or q - 1.  Quotients above
+// 2^15 (int8 path with Z < 256: rows with few valid keys) take the plain divide.
+template <bool U16, bool CLB>
+__device__ __forceinline__ uint32_t reciprocal(uint32_t Z) {
+    constexpr uint32_t Tp = U16 ? kTprimeU16 : kTprimeU8;
+    if (CLB) return Tp >> (31 - __clz((int)Z));
+    if (!U16 && Z < 256u) return Tp / Z;
+    constexpr float kScaled = U16 ? 32766.96875f : 8355832.0f;   // T' * (1 - 2^-20), exact in fp32
+    float rz;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rz) : "f"(__uint2float_rz(Z)));
+    const uint32_t q = __float2uint_rz(__fmul_rz(kScaled, rz));
+    const uint32_t rem = Tp - q * Z;
+    return q + (rem >= Z ? 1u : 0u);
+}
+
+// Number of valid keys of query i (a prefix of the row).
+template <bool CAUSAL>
+__device__ __forceinline__ int valid_keys(uint32_t i, const RowArgs &a) {
+    if (!CAUSAL) return a.Lk;
+    int nv = (int)i + a.causal_off + 1;
+    return min(max(nv, 0), a.Lk);
+}
+
+}  // namespace hccs

@@ -56,6 +56,9 @@ struct FusedArgs {
 // Launchers.  Each returns the CUDA error of the launch and adds to *launches.
 cudaError_t launch_rows(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                         cudaStream_t stream, uint64_t *launches);
+// Register-resident split-lane kernel (hccs_rows_split.cu): *taken tells whether the shape fit.
+cudaError_t try_launch_split(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                             cudaStream_t stream, bool *taken);
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches);
 bool fused_shape_supported(int32_t L, int32_t d);
 

@@ -21,43 +21,12 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "hccs_device.cuh"
 #include "hccs_internal.h"
 
 namespace hccs {
 
 namespace {
-
-constexpr uint32_t kTprimeU8 = 255u << 15;   // 255 * 2^R, R = INV_SHIFT = 15 (Eq. 8)
-constexpr uint32_t kTprimeU16 = 32767u;      // T for int16 output (Eq. 6)
-
-__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv &f) {
-    return (__umulhi(n, f.mul) + n) >> f.shift;
-}
-
-// (head, query index) of flat row r: head = (r / Lq) mod H, i = r mod Lq.
-__device__ __forceinline__ void row_coords(uint32_t r, const RowArgs &a, uint32_t &head, uint32_t &i) {
-    uint32_t bh = fast_div(r, a.div_Lq);
-    i = r - bh * (uint32_t)a.Lq;
-    bh += (uint32_t)a.slice0;
-    uint32_t b = fast_div(bh, a.div_H);
-    head = bh - b * (uint32_t)a.H;
-}
-
-// Step 5 of the kernel overview: the one scalar operation per row.
-template <bool U16, bool CLB>
-__device__ __forceinline__ uint32_t reciprocal(uint32_t Z) {
-    constexpr uint32_t Tp = U16 ? kTprimeU16 : kTprimeU8;
-    if (CLB) return Tp >> (31 - __clz((int)Z));   // k = floor(log2 Z), Eq. 9
-    return Tp / Z;                                  // Eq. 6 / Eq. 8
-}
-
-// Number of valid keys of query i (a prefix of the row).
-template <bool CAUSAL>
-__device__ __forceinline__ int valid_keys(uint32_t i, const RowArgs &a) {
-    if (!CAUSAL) return a.Lk;
-    int nv = (int)i + a.causal_off + 1;
-    return min(max(nv, 0), a.Lk);
-}
 
 // ------------------------------------------------------------------------------------------
 // Generic kernel: one warp per row, byte accesses, three passes over the (cached) row.
@@ -297,6 +266,12 @@ template <bool U16, bool CLB, bool CAUSAL>
 cudaError_t launch_mode(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
     const bool aligned = (((uintptr_t)x | (uintptr_t)p) & 15u) == 0 && a.Lk % 16 == 0;
     const bool shift_ok = U16 || a.out_shift <= 1;
+    if (aligned && shift_ok) {
+        bool taken = false;
+        cudaError_t e = try_launch_split(x, p, a, (U16 ? 1u : 0u) | (CLB ? 2u : 0u) | (CAUSAL ? 4u : 0u), st,
+                                         &taken);
+        if (taken) return e;
+    }
     if (aligned && shift_ok && a.Lk <= 1024) return launch_lanegroup<U16, CLB, CAUSAL>(x, p, a, st);
     return launch_generic<U16, CLB, CAUSAL>(x, p, a, st);
 }

@@ -1,0 +1,250 @@
+// Register-resident row kernel for Lk = 32*G*V (G lanes per row, V 32-byte chunks per lane):
+// Lk = 32, 64, 128, ..., 2048.  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
+//
+// Why 16-bit pairs: on sm_100a the byte-wise SIMD min/max intrinsics are emulated (about ten
+// instructions each), while min/max on s16x2 and the three-operand forms max(a+b, c) are single
+// instructions.  Each 32-bit word of four int8 logits is therefore split once into two words of
+// two sign-extended 16-bit lanes (bytes 0,2 and bytes 1,3; one PRMT each), and every later stage
+// works on those:
+//   stage 1  m = max x                      one max.s16x2 per split word
+//   stage 2+3  instead of delta = min(m - x, D) the kernel keeps the "closeness"
+//            r = D - delta = max(x + (D - m), 0)   one viaddmax.s16x2 per split word
+//            so that the score is s = B - S*delta = F + S*r with F = B - S*D (Eq. 2, Eq. 3);
+//            every quantity stays non-negative
+//   stage 4  Z = n_valid*F + S*sum(r)       one three-input add per word (16-bit lane sums)
+//   stage 5  rho once per row; p = (F*rho' + S*rho'*r) >> 16 with rho' = rho << (1 - OUT_SHIFT)
+// For uint8 output two elements share one 32x32->64-bit multiply-add: the operand r_a + r_b*2^24
+// times S*rho' plus F*rho'*(1 + 2^24) gives X_a + X_b*2^24 with both X < 2^24 (X = s*rho' <=
+// 255*2^16 because s <= Z), so p_a is byte 2 of the low word and p_b byte 1 of the high word.
+// For uint16 output one 32-bit multiply-add handles a pair directly (s*rho < 2^16).
+//
+// Causal rows: masked bytes are replaced by -128 right after the load (they can then never raise
+// the max), their closeness r_m = max(D - m - 128, 0) is subtracted from the sum in closed form,
+// and the output words are masked; the byte masks come from a small shared-memory table.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hccs_device.cuh"
+#include "hccs_internal.h"
+
+namespace hccs {
+
+namespace {
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+__device__ __forceinline__ void ldg256(const void *p, uint32_t (&r)[8]) {
+    asm volatile("ld.global.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+                   "=r"(r[7])
+                 : "l"(p));
+}
+
+__device__ __forceinline__ void stg256(void *p, const uint32_t (&r)[8]) {
+    asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
+__device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
+    uint64_t d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+
+constexpr uint32_t kSelEven = 0xA280u;   // bytes 0 and 2, each sign-extended to 16 bits
+constexpr uint32_t kSelOdd = 0xB391u;    // bytes 1 and 3, each sign-extended to 16 bits
+constexpr uint32_t kSelWide = 0x2440u;   // 16-bit pair (r_a, r_b) -> r_a + r_b * 2^24
+constexpr uint32_t kMinus128x4 = 0x80808080u;
+
+template <int G, int V, bool U16, bool CLB, bool CAUSAL>
+__global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, void *p_all, RowArgs a) {
+    constexpr int RW = 32 / G;      // rows per warp
+    constexpr int NW = 8 * V;       // 32-bit words of logits per lane
+    __shared__ uint32_t mask_tab[CAUSAL ? 33 * 8 : 1];   // [valid bytes of a chunk][word] -> byte mask
+    if (CAUSAL) {
+        for (int idx = threadIdx.x; idx < 33 * 8; idx += blockDim.x) {
+            const int nb = idx / 8 - 4 * (idx % 8);
+            mask_tab[idx] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
+        }
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % G;
+    const uint32_t row = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RW + lane / G;
+    const bool live = row < (uint32_t)a.rows;
+    uint32_t head = 0, qi = 0;
+    if (live) row_coords(row, a, head, qi);
+    const int nv = live ? valid_keys<CAUSAL>(qi, a) : 0;
+    const HeadEntry th = a.table[head];
+
+    // ---- loads: V independent 32-byte requests per lane
+    uint32_t e[NW], o[NW];          // first the raw words (in e), then the split lanes
+    int cnt[V];
+    const int8_t *x_row = x_all + (int64_t)row * a.Lk;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int col = (sub + v * G) * 32;
+        cnt[v] = CAUSAL ? min(max(nv - col, 0), 32) : (live ? 32 : 0);
+        uint32_t w[8];
+        if (cnt[v] > 0) {
+            ldg256(x_row + col, w);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) w[k] = kMinus128x4;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) e[8 * v + k] = w[k];
+    }
+
+    // ---- split into 16-bit lanes; stage 1: row max
+    uint32_t M = 0x80008000u;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t w = e[8 * v + k];
+            if (CAUSAL) {
+                const uint32_t bm = mask_tab[cnt[v] * 8 + k];
+                w = (w & bm) | (kMinus128x4 & ~bm);
+            }
+            const uint32_t ev = prmt(w, 0, kSelEven), od = prmt(w, 0, kSelOdd);
+            e[8 * v + k] = ev;
+            o[8 * v + k] = od;
+            M = __vmaxs2(M, __vmaxs2(ev, od));
+        }
+    }
+    int m = max((int)(short)(M & 0xffffu), (int)M >> 16);
+#pragma unroll
+    for (int s = G / 2; s; s >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, s));
+
+    // ---- stages 2-4: closeness r = max(x + (D - m), 0) and its row sum
+    const int cm = th.D - m;                               // in [-126, 255]
+    const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);    // (cm, cm) as 16-bit lanes
+    uint32_t rsum2 = 0;
+#pragma unroll
+    for (int k = 0; k < NW; ++k) {
+        e[k] = __viaddmax_s16x2(e[k], c2, 0u);
+        o[k] = __viaddmax_s16x2(o[k], c2, 0u);
+        rsum2 = rsum2 + e[k] + o[k];                       // lane sums stay below 2^16
+    }
+    int rsum = (int)(rsum2 & 0xffffu) + (int)(rsum2 >> 16);
+#pragma unroll
+    for (int s = G / 2; s; s >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, s);
+    if (CAUSAL) rsum -= (a.Lk - nv) * max(cm - 128, 0);    // masked keys were counted at x = -128
+    const int F = th.B - th.S * th.D;                      // floor score
+    const uint32_t Z = (uint32_t)(nv * F + th.S * rsum);
+    const uint32_t rho = reciprocal<U16, CLB>(max(Z, 1u));
+    if (!live) return;
+
+    // ---- stage 5: normalise and store
+    if (U16) {
+        const uint32_t a1 = (uint32_t)F * rho * 0x00010001u, b1 = (uint32_t)th.S * rho;
+        uint16_t *p_row = (uint16_t *)p_all + (int64_t)row * a.Lk;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int col = (sub + v * G) * 32;
+            uint32_t out[16];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t pe = e[8 * v + k] * b1 + a1, po = o[8 * v + k] * b1 + a1;
+                uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
+                if (CAUSAL) {
+                    const uint32_t bm = mask_tab[cnt[v] * 8 + k];
+                    q0 &= prmt(bm, 0, 0x1100u);
+                    q1 &= prmt(bm, 0, 0x3322u);
+                }
+                out[2 * k] = q0;
+                out[2 * k + 1] = q1;
+            }
+            uint32_t lo[8], hi[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { lo[k] = out[k]; hi[k] = out[8 + k]; }
+            stg256(p_row + col, lo);
+            stg256(p_row + col + 16, hi);
+        }
+    } else {
+        const int sh = 1 - a.out_shift;                    // 0 or 1 (checked by the launcher)
+        const uint32_t rp = rho << sh;
+        const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+        uint8_t *p_row = (uint8_t *)p_all + (int64_t)row * a.Lk;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int col = (sub + v * G) * 32;
+            uint32_t out[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                uint32_t q;
+                if (!CLB) {
+                    const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+                    const uint64_t pe = mad_wide(prmt(e[8 * v + k], 0, kSelWide), b1, A);
+                    const uint64_t po = mad_wide(prmt(o[8 * v + k], 0, kSelWide), b1, A);
+                    const uint32_t t0 = prmt((uint32_t)pe, (uint32_t)po, 0x0062u);
+                    const uint32_t t1 = prmt((uint32_t)(pe >> 32), (uint32_t)(po >> 32), 0x0051u);
+                    q = prmt(t0, t1, 0x5410u);
+                } else {
+                    // the leading-bit reciprocal can overshoot 255: saturate each element
+                    const uint32_t ev = e[8 * v + k], od = o[8 * v + k];
+                    const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
+                    const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
+                    const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
+                    const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
+                    q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                }
+                if (CAUSAL) q &= mask_tab[cnt[v] * 8 + k];
+                out[k] = q;
+            }
+            stg256(p_row + col, out);
+        }
+    }
+}
+
+template <int G, int V, bool U16, bool CLB, bool CAUSAL>
+cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
+    constexpr int ROWS_PER_CTA = 8 * (32 / G);
+    const unsigned blocks = (unsigned)(((int64_t)a.rows + ROWS_PER_CTA - 1) / ROWS_PER_CTA);
+    rows_split_kernel<G, V, U16, CLB, CAUSAL><<<blocks, 256, 0, st>>>(x, p, a);
+    return cudaGetLastError();
+}
+
+template <bool U16, bool CLB, bool CAUSAL>
+cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st, bool *taken) {
+    *taken = true;
+    switch (a.Lk) {
+        case 32: return launch_gv<1, 1, U16, CLB, CAUSAL>(x, p, a, st);
+        case 64: return launch_gv<1, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        case 128: return launch_gv<2, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        case 256: return launch_gv<4, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        case 512: return launch_gv<8, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        case 1024: return launch_gv<16, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        case 2048: return launch_gv<32, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        default: break;
+    }
+    *taken = false;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t try_launch_split(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                             cudaStream_t stream, bool *taken) {
+    *taken = false;
+    if ((((uintptr_t)logits | (uintptr_t)probs) & 31u) != 0) return cudaSuccess;
+    if (!(flags & 1u) && a.out_shift > 1) return cudaSuccess;
+    switch (flags & 7u) {
+        case 0: return launch_shape<false, false, false>(logits, probs, a, stream, taken);
+        case 1: return launch_shape<true, false, false>(logits, probs, a, stream, taken);
+        case 2: return launch_shape<false, true, false>(logits, probs, a, stream, taken);
+        case 3: return launch_shape<true, true, false>(logits, probs, a, stream, taken);
+        case 4: return launch_shape<false, false, true>(logits, probs, a, stream, taken);
+        case 5: return launch_shape<true, false, true>(logits, probs, a, stream, taken);
+        case 6: return launch_shape<false, true, true>(logits, probs, a, stream, taken);
+        default: return launch_shape<true, true, true>(logits, probs, a, stream, taken);
+    }
+}
+
+}  // namespace hccs

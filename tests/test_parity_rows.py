@@ -98,39 +98,43 @@ def test_many_heads_and_odd_head_count(ctx, oracle, hccs):
 
 
 def test_every_row_sum_is_reached(ctx, oracle, hccs):
-    """Rows built so that Z takes every value in 1..32767 (the exact divide per row is the one
-    scalar step): Lk = 16 with a table designed for 256 keys lets B start at 1."""
-    rows, thetas = [], []
-    # Z = nv*B - S*sum(delta): one key (nv = 1 through the causal mask) gives Z = B = 1..127
-    # 16 keys, S = 1: Z = 16*B - sum(delta), sum(delta) in 0..15*min(D, 255)
-    H = 127
-    x = np.zeros((1, H, 16, 16), dtype=np.int8)
-    theta = np.zeros((H, 3), dtype=np.int32)
-    rng = np.random.default_rng(1)
-    for h in range(H):
-        B = h + 1                       # n_design = 256: 1 <= B <= 127, floor score 1
-        D = max(1, min(127, B - 1))
-        theta[h] = (B, 1 if B - D >= 1 else 0, D)
-        x[0, h] = rng.integers(-128, 128, size=(16, 16))
-    wl = hccs.workloads.Workload("allZ-small", x.shape, 4, 256, theta, logits=x)
-    _check(ctx, oracle, wl, 4)
-    _check(ctx, oracle, wl, 5)
-    # large Z: Lk = 16, n_design = 16 -> B up to 2047; sweep sum(delta) through the row contents
-    H = 256
-    theta = np.zeros((H, 3), dtype=np.int32)
-    Bs = np.linspace(143, 2047, H).astype(np.int32)
-    theta[:, 0], theta[:, 1], theta[:, 2] = Bs, 1, 127
-    x = np.full((8, H, 16, 16), -128, dtype=np.int8)
-    x[..., 0] = 127                                     # the max; the others sit up to 255 below
-    steps = rng.integers(0, 128, size=(8, H, 16, 15))
-    x[..., 1:] = (127 - steps).astype(np.int8)
-    wl = hccs.workloads.Workload("allZ-large", x.shape, 0, 16, theta, logits=x)
-    seen = set()
+    """The reciprocal is the one scalar step per row and is computed without an integer divide,
+    so every row sum Z in 1..32767 is driven through it, in the byte kernel and in the fast one."""
+    W = hccs.workloads.Workload
+    # (a) one key per row, table designed for one key: Z = B for every B in 256..32767
+    Bs = np.arange(256, 32768, dtype=np.int32)
+    theta = np.stack([Bs, np.zeros_like(Bs), np.ones_like(Bs)], axis=1)
+    x = np.zeros((1, Bs.size, 1, 1), dtype=np.int8)
+    wl = W("allZ-one-key", x.shape, 0, 1, theta, logits=x)
     for flags in (0, 1):
         _check(ctx, oracle, wl, flags)
-    for b, h, i in np.ndindex(8, H, 16):
-        seen.add(int(16 * Bs[h] - np.minimum(127 - x[b, h, i].astype(int), 127).sum()))
-    assert len(seen) > 10000
+    # (b) Z below 256: a single valid key (causal row 0) of a table designed for 256 keys
+    H = 127
+    theta = np.array([(h + 1, 0, 1) for h in range(H)], dtype=np.int32)
+    rng = np.random.default_rng(1)
+    x = rng.integers(-128, 128, size=(1, H, 4, 64), dtype=np.int8)
+    wl = W("allZ-small", x.shape, 4, 256, theta, logits=x)
+    for flags in (4, 5, 6):
+        _check(ctx, oracle, wl, flags)
+    # (c) 64-key rows in the fast kernel: S = 1, D = 127, floor score F; a row whose closeness
+    # values r_j = 127 - (max - x_j) sum to R has Z = 64*F + R, R in 127..8128
+    Fs = [4, 129, 254, 379, 384]
+    theta = np.array([(F + 127, 1, 127) for F in Fs], dtype=np.int32)
+    R = np.arange(127, 8129)
+    x = np.full((1, len(Fs), R.size, 64), 0, dtype=np.int8)
+    rest = R - 127                                     # spread over the 63 other keys
+    base, extra = rest // 63, rest % 63
+    r = np.repeat(base[:, None], 63, axis=1)
+    r += (np.arange(63)[None, :] < extra[:, None])
+    assert r.max() <= 127 and (r.sum(axis=1) + 127 == R).all()
+    rows = np.concatenate([np.full((R.size, 1), 127), 127 - (127 - r)], axis=1)   # x_j = m - delta_j
+    rows[:, 1:] = 127 - (127 - r)
+    x[0, :] = rows.astype(np.int8)[None]
+    wl = W("allZ-64", x.shape, 0, 64, theta, logits=x)
+    for flags in (0, 1):
+        _check(ctx, oracle, wl, flags)
+    reached = {64 * F + int(v) for F in Fs for v in R}
+    assert set(range(383, 32705)) <= reached
 
 
 def test_empty_tensors_and_errors(ctx, hccs):
