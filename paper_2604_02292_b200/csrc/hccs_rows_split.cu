@@ -80,7 +80,20 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     uint32_t head = 0, qi = 0;
     if (live) row_coords(row, a, head, qi);
     const int nv = live ? valid_keys<CAUSAL>(qi, a) : 0;
+    // Programmatic dependent launch: everything above touches no global memory, so it may run
+    // while the previous kernel in the stream drains; all reads and writes come after the wait.
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const HeadEntry th = a.table[head];
+
+    // Causal: a chunk index v whose columns lie beyond every row of this warp is skipped
+    // altogether (warp-uniform), e.g. the right half of the first 64 queries of a 128-key head.
+    const int warp_nv = CAUSAL ? __reduce_max_sync(0xffffffffu, nv) : a.Lk;
+    auto chunk_used = [&](int v) { return !CAUSAL || v == 0 || v * G * 32 < warp_nv; };
+    int skipped_cols = 0;           // masked columns of this row that were never materialised
+#pragma unroll
+    for (int v = 1; v < V; ++v)
+        if (!chunk_used(v)) skipped_cols += 32 * G;
 
     // ---- loads: V independent 32-byte requests per lane
     uint32_t e[NW], o[NW];          // first the raw words (in e), then the split lanes
@@ -105,6 +118,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     uint32_t M = 0x80008000u;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
+        if (!chunk_used(v)) continue;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             uint32_t w = e[8 * v + k];
@@ -127,15 +141,20 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);    // (cm, cm) as 16-bit lanes
     uint32_t rsum2 = 0;
 #pragma unroll
-    for (int k = 0; k < NW; ++k) {
-        e[k] = __viaddmax_s16x2(e[k], c2, 0u);
-        o[k] = __viaddmax_s16x2(o[k], c2, 0u);
-        rsum2 = rsum2 + e[k] + o[k];                       // lane sums stay below 2^16
+    for (int v = 0; v < V; ++v) {
+        if (!chunk_used(v)) continue;
+#pragma unroll
+        for (int k = 8 * v; k < 8 * v + 8; ++k) {
+            e[k] = __viaddmax_s16x2(e[k], c2, 0u);
+            o[k] = __viaddmax_s16x2(o[k], c2, 0u);
+            rsum2 = rsum2 + e[k] + o[k];                   // lane sums stay below 2^16
+        }
     }
     int rsum = (int)(rsum2 & 0xffffu) + (int)(rsum2 >> 16);
 #pragma unroll
     for (int s = G / 2; s; s >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, s);
-    if (CAUSAL) rsum -= (a.Lk - nv) * max(cm - 128, 0);    // masked keys were counted at x = -128
+    // masked keys that were materialised were counted at x = -128
+    if (CAUSAL) rsum -= (a.Lk - nv - skipped_cols) * max(cm - 128, 0);
     const int F = th.B - th.S * th.D;                      // floor score
     const uint32_t Z = (uint32_t)(nv * F + th.S * rsum);
     const uint32_t rho = reciprocal<U16, CLB>(max(Z, 1u));
@@ -149,6 +168,10 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         for (int v = 0; v < V; ++v) {
             const int col = (sub + v * G) * 32;
             uint32_t out[16];
+            if (!chunk_used(v)) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) out[k] = 0;
+            } else
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const uint32_t pe = e[8 * v + k] * b1 + a1, po = o[8 * v + k] * b1 + a1;
@@ -176,6 +199,10 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         for (int v = 0; v < V; ++v) {
             const int col = (sub + v * G) * 32;
             uint32_t out[8];
+            if (!chunk_used(v)) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) out[k] = 0;
+            } else
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 uint32_t q;
@@ -183,9 +210,10 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                     const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
                     const uint64_t pe = mad_wide(prmt(e[8 * v + k], 0, kSelWide), b1, A);
                     const uint64_t po = mad_wide(prmt(o[8 * v + k], 0, kSelWide), b1, A);
-                    const uint32_t t0 = prmt((uint32_t)pe, (uint32_t)po, 0x0062u);
-                    const uint32_t t1 = prmt((uint32_t)(pe >> 32), (uint32_t)(po >> 32), 0x0051u);
-                    q = prmt(t0, t1, 0x5410u);
+                    // bytes 2,3 of the high words are zero: [p0,0,p2,0] + [0,p1,0,p3]
+                    const uint32_t t0 = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u);
+                    const uint32_t t1 = prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                    q = t0 + t1;
                 } else {
                     // the leading-bit reciprocal can overshoot 255: saturate each element
                     const uint32_t ev = e[8 * v + k], od = o[8 * v + k];
@@ -207,8 +235,16 @@ template <int G, int V, bool U16, bool CLB, bool CAUSAL>
 cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
     constexpr int ROWS_PER_CTA = 8 * (32 / G);
     const unsigned blocks = (unsigned)(((int64_t)a.rows + ROWS_PER_CTA - 1) / ROWS_PER_CTA);
-    rows_split_kernel<G, V, U16, CLB, CAUSAL><<<blocks, 256, 0, st>>>(x, p, a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL>, x, p, a);
 }
 
 template <bool U16, bool CLB, bool CAUSAL>
