@@ -18,7 +18,7 @@ struct hccs_ctx {
     int32_t num_heads = 0;                  // 0 = nothing uploaded
     int32_t n_design = 0;
     int32_t out_shift = 0;
-    uint32_t *d_status = nullptr;           // device status word
+    uint32_t *d_status = nullptr;           // device scratch: word 0 status, word 1 row counter
     uint32_t *h_status = nullptr;           // pinned landing place for it
     cudaEvent_t table_copied = nullptr;     // the staging buffers may be rewritten after this
     cudaEvent_t mult_copied = nullptr;
@@ -127,6 +127,7 @@ hccs::RowArgs make_row_args(const hccs_ctx *ctx, int32_t rows, int32_t H, int32_
     hccs::RowArgs a;
     a.table = ctx->d_table;
     a.status = ctx->d_status;
+    a.row_counter = ctx->d_status + 1;
     a.rows = rows;
     a.H = H;
     a.Lq = Lq;
@@ -154,8 +155,8 @@ hccs_status_t hccs_create(hccs_ctx_t **out, int device) {
     hccs_ctx *ctx = new (std::nothrow) hccs_ctx();
     if (!ctx) return HCCS_ERR_INVALID_ARG;
     ctx->device = device;
-    cudaError_t e = cudaMalloc(&ctx->d_status, sizeof(uint32_t));
-    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(uint32_t));
+    cudaError_t e = cudaMalloc(&ctx->d_status, 64 * sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 64 * sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaHostAlloc(&ctx->h_status, sizeof(uint32_t), cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->table_copied, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->mult_copied, cudaEventDisableTiming);
@@ -346,7 +347,7 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
     a.table = ctx->d_table;
     a.requant_mult = ctx->d_mult;
     a.status = ctx->d_status;
-    a.requant_shift = requant_shift;
+        a.requant_shift = requant_shift;
     a.B = B; a.H = H; a.L = L; a.d = d;
     a.out_shift = ctx->out_shift;
     a.flags = flags;

@@ -27,6 +27,7 @@ FastDiv make_fastdiv(uint32_t d);
 struct RowArgs {
     const HeadEntry *table;   // device, num_heads entries
     uint32_t *status;         // device status word (bounded waits report here)
+    uint32_t *row_counter;    // device scratch word: next row of the CTA-per-row kernel (zeroed per launch)
     int32_t rows;             // B*H*Lq
     int32_t H, Lq, Lk;
     int32_t causal_off;       // Lk - Lq
@@ -59,6 +60,9 @@ cudaError_t launch_rows(const int8_t *logits, void *probs, const RowArgs &a, uin
 // Register-resident split-lane kernel (hccs_rows_split.cu): *taken tells whether the shape fit.
 cudaError_t try_launch_split(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                              cudaStream_t stream, bool *taken);
+// CTA-per-row kernel for long rows (hccs_rows_cta.cu).
+cudaError_t try_launch_cta(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                           cudaStream_t stream, bool *taken);
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches);
 bool fused_shape_supported(int32_t L, int32_t d);
 

@@ -2,10 +2,12 @@
 //
 // Three kernels, all integer-only and bit-exact by construction (integer max and sum are
 // order-independent, so any reduction tree gives the one correct result):
-//   rows_lanegroup_kernel  Lk % 16 == 0, Lk <= 1024, 16-byte aligned: a group of G lanes owns
-//                          a row, each lane holds V 16-byte vectors of it in registers.
-//   rows_cta_kernel        Lk % 16 == 0, Lk > 1024: one CTA per row, the row staged in shared
-//                          memory by bulk asynchronous copies (TMA) behind an mbarrier.
+//   rows_split_kernel      (hccs_rows_split.cu) Lk = 32 ... 2048 in powers of two, 32-byte aligned:
+//                          the fast path.
+//   rows_lanegroup_kernel  other Lk % 16 == 0 up to 1024, 16-byte aligned: a group of G lanes
+//                          owns a row, each lane holds V 16-byte vectors of it in registers.
+//   rows_cta_kernel        (hccs_rows_cta.cu) longer rows with Lk % 16 == 0: one CTA per row, the
+//                          row staged in shared memory by bulk asynchronous copies (TMA).
 //   rows_generic_kernel    everything else (any Lk, any alignment): one warp per row, bytes.
 //
 // Word-parallel identities used by the fast kernels (all exact):
@@ -273,6 +275,12 @@ cudaError_t launch_mode(const int8_t *x, void *p, const RowArgs &a, cudaStream_t
         if (taken) return e;
     }
     if (aligned && shift_ok && a.Lk <= 1024) return launch_lanegroup<U16, CLB, CAUSAL>(x, p, a, st);
+    if (aligned) {
+        bool taken = false;
+        cudaError_t e = try_launch_cta(x, p, a, (U16 ? 1u : 0u) | (CLB ? 2u : 0u) | (CAUSAL ? 4u : 0u), st,
+                                       &taken);
+        if (taken) return e;
+    }
     return launch_generic<U16, CLB, CAUSAL>(x, p, a, st);
 }
 

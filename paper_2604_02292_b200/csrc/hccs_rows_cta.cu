@@ -1,0 +1,348 @@
+// CTA-per-row kernel for long rows (Lk % 16 == 0, up to 32752 keys): Algorithm 1 with the row
+// staged in shared memory.
+//
+// Persistent CTAs take rows from a global counter (rows cost different amounts of work under a
+// causal mask).  For every row one thread issues a 1-D bulk asynchronous copy (TMA,
+// cp.async.bulk) of the row's valid prefix into one of two shared-memory stages; the copy of
+// the next row is in flight while the CTA makes its three passes over the current one:
+//   pass 1  row max (Eq. 1)            pass 2  sum of the clamped scores (Eq. 2, 3, 5)
+//   once    reciprocal (Eq. 6 / 8 / 9) pass 3  normalise (Eq. 7 / int8 output path) into an
+//                                              output stage, written back by a bulk store.
+// The element arithmetic is the same 16-bit-pair formulation as the register-resident kernel.
+// Every wait on an mbarrier is bounded: when it runs out the CTA records
+// STATUS_ROW_TMA_TIMEOUT in the status word and stops taking rows.  No multicast, no clusters.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hccs_device.cuh"
+#include "hccs_internal.h"
+
+namespace hccs {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr long long kWaitCycles = 2000000000ll;   // about one second of SM clocks: then a wait is given up
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
+    uint64_t d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem),
+                 "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_all() {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t byte_prefix_mask(int nb) {
+    return nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
+}
+
+__device__ __forceinline__ int block_reduce(int v, bool is_max, int *scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int s = 16; s; s >>= 1) {
+        const int other = __shfl_xor_sync(0xffffffffu, v, s);
+        v = is_max ? max(v, other) : v + other;
+    }
+    __syncthreads();                       // the previous user of scratch is done
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    int r = scratch[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) r = is_max ? max(r, scratch[w]) : r + scratch[w];
+    return r;
+}
+
+struct RowJob {
+    int32_t row;        // -1: no more rows
+    int32_t nv;         // valid keys
+    uint32_t head;
+    uint32_t bytes;     // bytes to copy in (nv rounded up to 16)
+};
+
+template <bool U16, bool CLB, bool CAUSAL>
+__global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all, void *p_all, RowArgs a) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    // layout: [stage 0 | stage 1 | output stage], each Lk (output: Lk * element size) bytes
+    uint8_t *in_stage[2] = {smem, smem + a.Lk};
+    uint8_t *out_stage = smem + 2 * a.Lk;
+    __shared__ __align__(8) uint64_t full_bar[2];
+    __shared__ RowJob job[2];
+    __shared__ int red[kThreads / 32];
+    const int tid = threadIdx.x;
+    const uint32_t bar[2] = {smem_u32(&full_bar[0]), smem_u32(&full_bar[1])};
+
+    // thread 0: take the next row from the counter and start its copy into stage s
+    auto fetch = [&](int s) {
+        RowJob j;
+        j.row = (int32_t)atomicAdd(a.row_counter, 1u);
+        j.nv = 0; j.head = 0; j.bytes = 0;
+        if (j.row >= a.rows) {
+            j.row = -1;
+        } else {
+            uint32_t qi;
+            row_coords((uint32_t)j.row, a, j.head, qi);
+            j.nv = valid_keys<CAUSAL>(qi, a);
+            j.bytes = (uint32_t)((j.nv + 15) & ~15);
+            if (j.bytes) {
+                mbar_expect_tx(bar[s], j.bytes);
+                bulk_load(smem_u32(in_stage[s]), x_all + (int64_t)j.row * a.Lk, j.bytes, bar[s]);
+            }
+        }
+        job[s] = j;
+    };
+
+    if (tid == 0) {
+        mbar_init(bar[0], 1);
+        mbar_init(bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fetch(0);
+    }
+    __syncthreads();
+
+    uint32_t phase[2] = {0, 0};
+    const int osz = U16 ? 2 : 1;
+    for (int it = 0;; ++it) {
+        const int s = it & 1;
+        // stage s^1 was consumed in the previous iteration (all threads passed its last barrier)
+        if (tid == 0) fetch(s ^ 1);
+        const RowJob j = job[s];
+        if (j.row < 0) break;
+        bool ok = true;
+        if (j.bytes) {
+            ok = mbar_wait(bar[s], phase[s]);
+            phase[s] ^= 1;
+        }
+        if (!__syncthreads_and(ok)) {                 // uniform decision: give up together
+            if (tid == 0) {
+                atomicOr(a.status, STATUS_ROW_TMA_TIMEOUT);
+                // give the copy that was started for the other stage a bounded chance to land
+                if (job[s ^ 1].row >= 0 && job[s ^ 1].bytes) (void)mbar_wait(bar[s ^ 1], phase[s ^ 1]);
+            }
+            break;
+        }
+        const HeadEntry th = a.table[j.head];
+        const uint8_t *xin = in_stage[s];
+        const int nvec = (int)(j.bytes >> 4);         // 16-byte vectors that hold valid keys
+
+        // ---- pass 1: row max
+        uint32_t M = 0x80008000u;
+        for (int v = tid; v < nvec; v += kThreads) {
+            const uint4 w4 = *reinterpret_cast<const uint4 *>(xin + 16 * v);
+            uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (CAUSAL) {
+                    const uint32_t bm = byte_prefix_mask(j.nv - 16 * v - 4 * k);
+                    w[k] = (w[k] & bm) | (0x80808080u & ~bm);
+                }
+                M = __vmaxs2(M, __vmaxs2(prmt(w[k], 0, 0xA280u), prmt(w[k], 0, 0xB391u)));
+            }
+        }
+        const int m = block_reduce(max((int)(short)(M & 0xffffu), (int)M >> 16), true, red);
+
+        // ---- pass 2: sum of the closeness values r = max(x + (D - m), 0) over the valid keys
+        const int cm = th.D - m;
+        const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
+        uint32_t rsum2 = 0;
+        for (int v = tid; v < nvec; v += kThreads) {
+            const uint4 w4 = *reinterpret_cast<const uint4 *>(xin + 16 * v);
+            uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
+                uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                if (CAUSAL) {
+                    const uint32_t bm = byte_prefix_mask(j.nv - 16 * v - 4 * k);
+                    ev &= prmt(bm, 0, 0x2200u);       // 16-bit lane masks of bytes 0,2 / 1,3
+                    od &= prmt(bm, 0, 0x3311u);
+                }
+                rsum2 += ev + od;                     // at most 8 vectors per thread: no overflow
+            }
+        }
+        const int rsum = block_reduce((int)(rsum2 & 0xffffu) + (int)(rsum2 >> 16), false, red);
+        const int F = th.B - th.S * th.D;
+        const uint32_t Z = (uint32_t)(j.nv * F + th.S * rsum);
+        const uint32_t rho = reciprocal<U16, CLB>(max(Z, 1u));
+
+        // ---- the output stage may still be read by the previous row's bulk store
+        if (tid == 0) bulk_store_wait_read();
+        __syncthreads();
+
+        // ---- pass 3: normalise into the output stage
+        const int total_vec = a.Lk >> 4;
+        if (U16) {
+            const uint32_t a1 = (uint32_t)F * rho * 0x00010001u, b1 = (uint32_t)th.S * rho;
+            for (int v = tid; v < total_vec; v += kThreads) {
+                uint32_t o[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                if (v < nvec) {
+                    const uint4 w4 = *reinterpret_cast<const uint4 *>(xin + 16 * v);
+                    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t pe = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u) * b1 + a1;
+                        const uint32_t po = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u) * b1 + a1;
+                        uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
+                        if (CAUSAL) {
+                            const uint32_t bm = byte_prefix_mask(j.nv - 16 * v - 4 * k);
+                            q0 &= prmt(bm, 0, 0x1100u);
+                            q1 &= prmt(bm, 0, 0x3322u);
+                        }
+                        o[2 * k] = q0;
+                        o[2 * k + 1] = q1;
+                    }
+                }
+                uint4 *dst = reinterpret_cast<uint4 *>(out_stage + 32 * v);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+        } else if (a.out_shift <= 1) {
+            const uint32_t rp = rho << (1 - a.out_shift);
+            const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+            for (int v = tid; v < total_vec; v += kThreads) {
+                uint32_t o[4] = {0, 0, 0, 0};
+                if (v < nvec) {
+                    const uint4 w4 = *reinterpret_cast<const uint4 *>(xin + 16 * v);
+                    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
+                        const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                        uint32_t q;
+                        if (!CLB) {
+                            const uint64_t pe = mad_wide(prmt(ev, 0, 0x2440u), b1, A);
+                            const uint64_t po = mad_wide(prmt(od, 0, 0x2440u), b1, A);
+                            q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) +
+                                prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                        } else {
+                            const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
+                            const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
+                            const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
+                            const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
+                            q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                        }
+                        if (CAUSAL) q &= byte_prefix_mask(j.nv - 16 * v - 4 * k);
+                        o[k] = q;
+                    }
+                }
+                *reinterpret_cast<uint4 *>(out_stage + 16 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        } else {
+            // OUT_SHIFT >= 2: the result is not byte-aligned in the product; shift each element
+            const uint32_t a1 = (uint32_t)F * rho, b1 = (uint32_t)th.S * rho;
+            const int sh = 15 + a.out_shift;
+            for (int v = tid; v < total_vec; v += kThreads) {
+                uint32_t o[4] = {0, 0, 0, 0};
+                if (v < nvec) {
+                    const uint4 w4 = *reinterpret_cast<const uint4 *>(xin + 16 * v);
+                    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
+                        const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                        const uint32_t x0 = min((a1 + b1 * (ev & 0xffffu)) >> sh, 255u);
+                        const uint32_t x1 = min((a1 + b1 * (od & 0xffffu)) >> sh, 255u);
+                        const uint32_t x2 = min((a1 + b1 * (ev >> 16)) >> sh, 255u);
+                        const uint32_t x3 = min((a1 + b1 * (od >> 16)) >> sh, 255u);
+                        uint32_t q = x0 | (x1 << 8) | (x2 << 16) | (x3 << 24);
+                        if (CAUSAL) q &= byte_prefix_mask(j.nv - 16 * v - 4 * k);
+                        o[k] = q;
+                    }
+                }
+                *reinterpret_cast<uint4 *>(out_stage + 16 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        // make the generic-proxy writes visible to the bulk store, then hand the row over
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0)
+            bulk_store((uint8_t *)p_all + (int64_t)j.row * a.Lk * osz, smem_u32(out_stage),
+                       (uint32_t)(a.Lk * osz));
+    }
+    if (tid == 0) bulk_store_wait_all();   // shared memory must outlive the last store
+}
+
+template <bool U16, bool CLB, bool CAUSAL>
+cudaError_t launch_cta(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
+    const size_t smem = (size_t)a.Lk * (U16 ? 4 : 3);
+    auto kernel = rows_cta_kernel<U16, CLB, CAUSAL>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(a.row_counter, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return e;
+    int ctas_per_sm = (int)((200u * 1024u) / (smem + 1024));
+    if (ctas_per_sm < 1) ctas_per_sm = 1;
+    if (ctas_per_sm > 8) ctas_per_sm = 8;
+    int64_t blocks = (int64_t)148 * ctas_per_sm;
+    if (blocks > a.rows) blocks = a.rows;
+    kernel<<<(unsigned)blocks, kThreads, smem, st>>>(x, p, a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t try_launch_cta(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                           cudaStream_t stream, bool *taken) {
+    *taken = false;
+    if ((((uintptr_t)logits | (uintptr_t)probs) & 15u) != 0 || a.Lk % 16 != 0 || a.Lk < 256) return cudaSuccess;
+    *taken = true;
+    switch (flags & 7u) {
+        case 0: return launch_cta<false, false, false>(logits, probs, a, stream);
+        case 1: return launch_cta<true, false, false>(logits, probs, a, stream);
+        case 2: return launch_cta<false, true, false>(logits, probs, a, stream);
+        case 3: return launch_cta<true, true, false>(logits, probs, a, stream);
+        case 4: return launch_cta<false, false, true>(logits, probs, a, stream);
+        case 5: return launch_cta<true, false, true>(logits, probs, a, stream);
+        case 6: return launch_cta<false, true, true>(logits, probs, a, stream);
+        default: return launch_cta<true, true, true>(logits, probs, a, stream);
+    }
+}
+
+}  // namespace hccs

@@ -40,7 +40,7 @@ def test_reduced_configs_all_modes(ctx, oracle, hccs, c, batch, flags):
 # row lengths around every dispatch boundary: lane-group sizes, two vectors per lane, the
 # CTA-per-row kernel, ragged tails and lengths that are no multiple of 16
 LENGTHS = [1, 2, 3, 15, 16, 17, 31, 32, 33, 48, 64, 80, 96, 100, 112, 128, 144, 256, 257, 272, 384,
-           496, 512, 528, 1000, 1008, 1024, 1040, 2048, 2064, 4096, 5000, 8192]
+           496, 512, 528, 1000, 1008, 1024, 1040, 2048, 2064, 2304, 4096, 4112, 5000, 8192, 16384, 32752]
 
 
 @pytest.mark.parametrize("Lk", LENGTHS)
@@ -53,7 +53,8 @@ def test_row_lengths(ctx, oracle, hccs, Lk):
 
 
 @pytest.mark.parametrize("Lq,Lk", [(1, 64), (5, 64), (64, 5), (100, 128), (128, 100), (33, 512),
-                                   (40, 1024), (7, 2048), (3, 1), (130, 144), (2100, 2048)])
+                                   (40, 1024), (7, 2048), (3, 1), (130, 144), (2100, 2048), (300, 4096),
+                                   (4100, 4112)])
 def test_causal_alignment(ctx, oracle, hccs, Lq, Lk):
     for flags in (4, 5, 6, 7):
         wl = hccs.workloads.make_rows(50 + Lq + Lk, (2, 3, Lq, Lk), kind="gauss")
