@@ -160,6 +160,39 @@ const char *hccs_status_string(hccs_status_t status);
 /* Number of kernels launched through this context since creation (for launch accounting). */
 uint64_t hccs_launch_count(const hccs_ctx_t *ctx);
 
+/*
+ * hccs_forward for callers that are not allowed to allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a memory pool's or a
+ * framework's allocator callback, in a process whose device memory was handed out in full at
+ * start-up (a serving engine that pre-claims the whole GPU), or in a latency-critical loop where
+ * an allocation (which may synchronise the whole device) cannot be tolerated.  Such a caller
+ * cannot create an hccs_ctx_t, because the context allocates its parameter table.
+ *
+ * What it does: the same result as hccs_forward, computed by the shared-memory-staged
+ * one-CTA-per-row kernel, with all of the library's working memory (parameter table, the row
+ * counter of the persistent CTAs, the status word) in one fixed 4.25 KB array that is part of
+ * the loaded library image on every GPU.  No context, no cudaMalloc/cudaFree, no allocating
+ * library call; the tensors are the caller's.
+ *   params, num_heads, n_design, out_shift   HOST table, checked exactly as hccs_params_upload
+ *        does; num_heads above 256 does not fit the fixed array: HCCS_ERR_UNSUPPORTED
+ *   logits, probs, B, H, Lq, Lk, flags       as hccs_forward, on the CURRENT device; this entry
+ *        point needs Lk % 16 == 0 and 16-byte aligned pointers (else HCCS_ERR_UNSUPPORTED)
+ *   timed_out   NULL: fully asynchronous.  Non-NULL (host): the call synchronises `cuda_stream`
+ *        and stores the status word there; non-zero also returns HCCS_ERR_DEVICE_TIMEOUT.
+ * The first call on each device looks up the device address of the fixed array; make that
+ * first call outside any stream capture.  All calls on a device share the array and it keeps
+ * the previous call's contents: each call rewrites the table and clears the counter and status
+ * on `cuda_stream` before its kernel.  Two calls whose work overlaps on the GPU (different
+ * streams, no dependency between them) therefore race on it -- serialise them.
+ */
+hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *params, int32_t num_heads,
+                                          int32_t n_design, int32_t out_shift,
+                                          const int8_t *logits, void *probs,
+                                          int32_t B, int32_t H, int32_t Lq, int32_t Lk,
+                                          uint32_t flags, uint32_t *timed_out, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

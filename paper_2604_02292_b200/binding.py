@@ -37,7 +37,7 @@ HCCS_CAUSAL = 4
 
 EXPORTS = ("hccs_create", "hccs_destroy", "hccs_params_check", "hccs_params_upload", "hccs_forward", "hccs_forward_host",
            "hccs_attention_fused", "hccs_device_status", "hccs_last_cuda_error", "hccs_status_string",
-           "hccs_launch_count")
+           "hccs_launch_count", "hccs_forward_static_scratch")
 
 _vp, _i32, _u32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32
 
@@ -64,6 +64,11 @@ _lib.hccs_status_string.argtypes = [ctypes.c_int]
 _lib.hccs_status_string.restype = ctypes.c_char_p
 _lib.hccs_launch_count.argtypes = [_vp]
 _lib.hccs_launch_count.restype = ctypes.c_uint64
+
+
+_lib.hccs_forward_static_scratch.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _i32, _u32,
+                                             ctypes.POINTER(_u32), _vp]
+_lib.hccs_forward_static_scratch.restype = ctypes.c_int
 
 
 def hccs_status_string(status: int) -> str:
@@ -181,6 +186,25 @@ class Context:
 
     def hccs_launch_count(self) -> int:
         return int(_lib.hccs_launch_count(self._h))
+
+
+def hccs_forward_static_scratch(params, n_design: int, logits, probs, flags: int = 0, out_shift: int = 0,
+                                check_timeout: bool = False, stream=None) -> int:
+    """hccs_forward without a context and without any allocation inside the library: for callers
+    that may not allocate device memory.  Runs on the current device; ``logits``/``probs`` are the
+    caller's tensors.  With ``check_timeout`` the call synchronises and returns the status word."""
+    arr = np.ascontiguousarray(params, dtype=np.int32).reshape(-1, 3)
+    B, H, Lq, Lk = logits.shape
+    _check_tensor(logits, "logits", 1)
+    _check_tensor(probs, "probs", 2 if flags & HCCS_OUT_U16 else 1, logits.shape)
+    word = _u32(0)
+    st = _lib.hccs_forward_static_scratch(arr.ctypes.data_as(_vp), arr.shape[0], int(n_design),
+                                          int(out_shift), _ptr(logits), _ptr(probs), B, H, Lq, Lk,
+                                          int(flags), ctypes.byref(word) if check_timeout else None,
+                                          _stream_ptr(stream))
+    if st != HCCS_OK:
+        raise HccsError(st, "hccs_forward_static_scratch")
+    return int(word.value)
 
 
 def _check_tensor(t, name, itemsize, shape=None, device="cuda"):

@@ -346,3 +346,116 @@ cudaError_t try_launch_cta(const int8_t *logits, void *probs, const RowArgs &a, 
 }
 
 }  // namespace hccs
+
+// ------------------------------------------------------------------------------------------
+// hccs_forward_static_scratch: the CTA-per-row kernel for callers that must not allocate.
+// ------------------------------------------------------------------------------------------
+// Everything the kernel needs besides the caller's tensors lives in this one file-scope device
+// array, which every GPU that loads the library holds until the process exits:
+//   word 0            status word (bounded waits report here)
+//   word 1            row counter of the persistent CTAs
+//   from byte 256 on  the per-head parameter table, kStaticMaxHeads entries
+namespace {
+
+constexpr int kStaticMaxHeads = 256;
+constexpr int kStaticTableOffsetWords = 64;
+constexpr int kStaticWords = kStaticTableOffsetWords + kStaticMaxHeads * (int)(sizeof(hccs::HeadEntry) / 4);
+static __device__ __align__(256) uint32_t g_static_scratch[kStaticWords];
+
+constexpr int kStaticMaxDevices = 64;
+uint32_t *g_static_ptr[kStaticMaxDevices] = {};   // device address of the array, per device
+
+// The array's name is only a host-side handle; the address the kernel can use has to be asked
+// for, once per device and with that device current.
+cudaError_t static_scratch_address(int device, uint32_t **out) {
+    if (!g_static_ptr[device]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[device] = static_cast<uint32_t *>(p);
+    }
+    *out = g_static_ptr[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *params, int32_t num_heads,
+                                                     int32_t n_design, int32_t out_shift,
+                                                     const int8_t *logits, void *probs, int32_t B,
+                                                     int32_t H, int32_t Lq, int32_t Lk, uint32_t flags,
+                                                     uint32_t *timed_out, void *cuda_stream) {
+    if (timed_out) *timed_out = 0;
+    if (B < 0 || H < 0 || Lq < 0 || Lk < 0 || (flags & ~7u)) return HCCS_ERR_INVALID_ARG;
+    if (out_shift < 0 || out_shift > 8) return HCCS_ERR_INVALID_ARG;
+    hccs_status_t st = hccs_params_check(params, num_heads, n_design, nullptr);
+    if (st != HCCS_OK) return st;
+    if (H != num_heads) return HCCS_ERR_INVALID_ARG;
+    if (num_heads > kStaticMaxHeads) return HCCS_ERR_UNSUPPORTED;      // beyond the static table
+    if (Lk > n_design) return HCCS_ERR_CONSTRAINT;
+    const int64_t rows = (int64_t)B * H * Lq;
+    if (rows >= (1ll << 31)) return HCCS_ERR_UNSUPPORTED;
+    if (rows * Lk == 0) return HCCS_OK;
+    if (!logits || !probs) return HCCS_ERR_INVALID_ARG;
+    if (Lk % 16 != 0 || (((uintptr_t)logits | (uintptr_t)probs) & 15u) != 0) return HCCS_ERR_UNSUPPORTED;
+    if ((flags & HCCS_OUT_U16) && (const void *)logits == probs) return HCCS_ERR_INVALID_ARG;
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kStaticMaxDevices) {
+        (void)cudaGetLastError();
+        return HCCS_ERR_CUDA;
+    }
+    uint32_t *scratch = nullptr;
+    if (static_scratch_address(device, &scratch) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return HCCS_ERR_CUDA;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    // The array keeps whatever the previous call left: rewrite the table, clear the status
+    // word (the launcher clears the row counter).
+    hccs::HeadEntry table[kStaticMaxHeads];
+    for (int32_t h = 0; h < num_heads; ++h) {
+        table[h].B = params[h].B;
+        table[h].S = params[h].S;
+        table[h].D = params[h].Dmax;
+        table[h].Drep = (uint32_t)params[h].Dmax * 0x01010101u;
+    }
+    hccs::HeadEntry *d_table = reinterpret_cast<hccs::HeadEntry *>(scratch + kStaticTableOffsetWords);
+    cudaError_t e = cudaMemcpyAsync(d_table, table, sizeof(hccs::HeadEntry) * num_heads,
+                                    cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(scratch, 0, sizeof(uint32_t), stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return HCCS_ERR_CUDA; }
+
+    hccs::RowArgs a;
+    a.table = d_table;
+    a.status = scratch;
+    a.row_counter = scratch + 1;
+    a.rows = (int32_t)rows;
+    a.H = H;
+    a.Lq = Lq;
+    a.Lk = Lk;
+    a.causal_off = Lk - Lq;
+    a.out_shift = out_shift;
+    a.slice0 = 0;
+    a.div_Lq = hccs::make_fastdiv((uint32_t)Lq);
+    a.div_H = hccs::make_fastdiv((uint32_t)H);
+    switch (flags & 7u) {
+        case 0: e = hccs::launch_cta<false, false, false>(logits, probs, a, stream); break;
+        case 1: e = hccs::launch_cta<true, false, false>(logits, probs, a, stream); break;
+        case 2: e = hccs::launch_cta<false, true, false>(logits, probs, a, stream); break;
+        case 3: e = hccs::launch_cta<true, true, false>(logits, probs, a, stream); break;
+        case 4: e = hccs::launch_cta<false, false, true>(logits, probs, a, stream); break;
+        case 5: e = hccs::launch_cta<true, false, true>(logits, probs, a, stream); break;
+        case 6: e = hccs::launch_cta<false, true, true>(logits, probs, a, stream); break;
+        default: e = hccs::launch_cta<true, true, true>(logits, probs, a, stream); break;
+    }
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return HCCS_ERR_CUDA; }
+    if (timed_out) {
+        e = cudaMemcpyAsync(timed_out, scratch, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return HCCS_ERR_CUDA; }
+        if (*timed_out) return HCCS_ERR_DEVICE_TIMEOUT;
+    }
+    return HCCS_OK;
+}
