@@ -328,6 +328,9 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
     if (requant_shift < 1 || requant_shift > 31) return HCCS_ERR_INVALID_ARG;
     for (int32_t h = 0; h < H; ++h)
         if (requant_mult[h] < 0 || requant_mult[h] >= (1 << 13)) return HCCS_ERR_INVALID_ARG;
+    // the kernel requantises with the multiplier pre-shifted by 32 - requant_shift bits
+    for (int32_t h = 0; h < H; ++h)
+        if ((int64_t)requant_mult[h] << (32 - requant_shift) >= (1ll << 31)) return HCCS_ERR_UNSUPPORTED;
     if (L > ctx->n_design) return HCCS_ERR_CONSTRAINT;
     if ((int64_t)B * H * L * d == 0) return HCCS_OK;
     if (!Q || !K || !V || !O) return HCCS_ERR_INVALID_ARG;

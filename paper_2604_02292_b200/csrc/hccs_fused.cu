@@ -1,7 +1,451 @@
-// Fused int8 attention (placeholder translation unit until the tcgen05 kernel lands).
+// Fused int8 attention for one (batch, head, 128-query tile) per CTA:
+//     S = Q.K^T (int32)  ->  x = requantise(S) (int8)  ->  P = HCCS(x) (uint8)  ->  O = P.V (int32)
+// The two contractions run on the 5th-generation tensor cores (tcgen05.mma kind::i8, operands in
+// shared memory staged by TMA, accumulators in tensor memory); the softmax surrogate itself is
+// plain integer ALU work (Algorithm 1 of the paper) done by the thread that owns the row.
+//
+// Why it is organised this way:
+//   * HCCS needs the whole row before it can normalise (the clamp makes the usual online
+//     rescaling of exp-softmax impossible), so the CTA keeps the full 128 x L int8 logit panel in
+//     shared memory (128 KB at L = 1024).  The panel is laid out as the K-major, 128-byte-swizzled
+//     operand the second contraction wants, so P is produced in place and never moves.
+//   * tcgen05.ld with the 32x32b shape gives thread t of the four row warps TMEM lane t, i.e. one
+//     query row with all its keys: max, sum, reciprocal and normalisation need no cross-thread
+//     reduction at all.
+//   * K tiles are consumed during the first contraction only and V tiles during the second, so V
+//     is loaded into the buffer K occupied, while the row warps do the HCCS passes.
+//   * V is used as stored ([key][64], keys outermost): that is exactly the MN-major, 64-byte
+//     swizzled B operand, so no transposition is needed.
+//
+// Warp roles (160 threads): warps 0-3 own the 128 rows (TMEM lane quarter = warp index); warp 4
+// lane 0 issues every TMA copy and every MMA.  All mbarrier waits are bounded; a wait that runs
+// out sets STATUS_FUSED_TIMEOUT, raises an abort flag that every other wait observes, and the CTA
+// leaves through the common exit, which frees its tensor memory.  No clusters, no multicast.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hccs_device.cuh"
 #include "hccs_internal.h"
 
 namespace hccs {
-bool fused_shape_supported(int32_t, int32_t) { return false; }
-cudaError_t launch_fused(const FusedArgs &, cudaStream_t, uint64_t *) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kRowThreads = 128;
+constexpr int kThreads = 160;
+constexpr int kD = 64;                    // head dimension (bytes per Q/K/V row)
+constexpr int kTile = 128;                // queries per CTA, keys per block
+constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
+constexpr int kPanelBlockBytes = kTile * 128;   // 16 KB: 128 rows x 128 keys of the panel
+constexpr int kMaxBlocks = 8;             // L <= 1024
+constexpr uint32_t kTmemCols = 512;       // S0 [0,128)  S1 [128,256)  O [256,320)
+constexpr long long kWaitCycles = 2000000000ll;
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint64_t mad_wide_u32(uint32_t a, uint32_t b, uint64_t c) {
+    uint64_t d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ int64_t mad_wide_s32(int32_t a, int32_t b, int64_t c) {
+    int64_t d;
+    asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded, abort-aware wait.  Returns false when the wait was given up (here or elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          uint32_t *status) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicOr(status, STATUS_FUSED_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], int8 operands, int32 accumulator.
+__device__ __forceinline__ void tcgen05_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---------------------------------------------------------------- descriptors
+// Shared-memory matrix descriptor: start address, leading/stride byte offsets (all >> 4), the
+// Blackwell version field (1 at bit 46) and the swizzle mode in bits [61,64).
+constexpr uint64_t kSwizzle128 = 2, kSwizzle64 = 4;
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint64_t swizzle) {
+    return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | (swizzle << 61);
+}
+// Instruction descriptor of kind::i8: D = int32 (2 at bit 4), operand formats at bits 7 and 10
+// (0 = uint8, 1 = int8), B MN-major flag at bit 16, N >> 3 at bit 17, M >> 4 at bit 24.
+constexpr uint32_t instr_desc(uint32_t a_signed, uint32_t b_signed, uint32_t b_mn_major, uint32_t M, uint32_t N) {
+    return (2u << 4) | (a_signed << 7) | (b_signed << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+constexpr uint32_t kIdescQK = instr_desc(1, 1, 0, 128, 128);   // S = Q.K^T : int8 x int8, both K-major
+constexpr uint32_t kIdescPV = instr_desc(0, 1, 1, 128, 64);    // O = P.V   : uint8 x int8, V MN-major
+
+struct FusedSmemBarriers {
+    uint64_t q_full;
+    uint64_t k_full[kMaxBlocks];
+    uint64_t k_done;        // every MMA of the first contraction has finished reading K
+    uint64_t v_full;
+    uint64_t s_full[2];
+    uint64_t s_free[2];
+    uint64_t p_ready;
+    uint64_t o_full;
+};
+
+template <bool CLB, bool CAUSAL>
+__global__ void __launch_bounds__(kThreads, 1)
+fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v, FusedArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) FusedSmemBarriers bars;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nblk = a.L / kTile;                         // key blocks (and query tiles) per head
+    const int bh = blockIdx.x / nblk, qt = blockIdx.x % nblk;
+    const int head = bh % a.H;
+    const int q0 = qt * kTile;
+    const int kblocks = CAUSAL ? qt + 1 : nblk;           // key blocks this tile needs
+    volatile int *abortp = &abort_flag;
+
+    // shared-memory carve-up (1024-byte aligned: required by the swizzled layouts)
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t s_q = base;                                            // Q tile
+    const uint32_t s_kv = base + kTileBytes;                              // K tiles, later V tiles
+    const uint32_t s_p = s_kv + (uint32_t)nblk * kTileBytes;              // logit / probability panel
+    uint8_t *panel = gen_base + kTileBytes + (size_t)nblk * kTileBytes;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bars.q_full), 1);
+        for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.k_full[i]), 1);
+        mbar_init(smem_u32(&bars.k_done), 1);
+        mbar_init(smem_u32(&bars.v_full), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&bars.s_full[i]), 1);
+            mbar_init(smem_u32(&bars.s_free[i]), kRowThreads);
+        }
+        mbar_init(smem_u32(&bars.p_ready), kRowThreads);
+        mbar_init(smem_u32(&bars.o_full), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 4) {   // one warp allocates the tensor memory for the CTA
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+
+    if (warp == 4) {
+        // ===================================================== control thread: TMA + MMA issue
+        if (lane == 0) {
+            bool ok = true;
+            mbar_expect_tx(smem_u32(&bars.q_full), kTileBytes);
+            tma_load_2d(s_q, &map_q, 0, bh * a.L + q0, smem_u32(&bars.q_full));
+            for (int kb = 0; kb < kblocks; ++kb) {
+                mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
+                tma_load_2d(s_kv + kb * kTileBytes, &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
+            }
+            ok = mbar_wait(smem_u32(&bars.q_full), 0, abortp, a.status);
+            // ---- first contraction: S_kb = Q . K_kb^T, two k-steps of 32 over d = 64
+            for (int kb = 0; ok && kb < kblocks; ++kb) {
+                const int sb = kb & 1;
+                if (kb >= 2) ok = mbar_wait(smem_u32(&bars.s_free[sb]), ((kb >> 1) - 1) & 1, abortp, a.status);
+                if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), 0, abortp, a.status);
+                if (!ok) break;
+                tcgen05_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 2; ++ks) {
+                    const uint64_t da = smem_desc(s_q + ks * 32, 16, 512, kSwizzle64);
+                    const uint64_t db = smem_desc(s_kv + kb * kTileBytes + ks * 32, 16, 512, kSwizzle64);
+                    tcgen05_mma_i8(tmem + sb * 128, da, db, kIdescQK, ks);
+                }
+                tcgen05_commit(smem_u32(&bars.s_full[sb]));
+            }
+            if (ok) {
+                tcgen05_commit(smem_u32(&bars.k_done));
+                ok = mbar_wait(smem_u32(&bars.k_done), 0, abortp, a.status);
+            }
+            // ---- V replaces K in shared memory while the row warps run the softmax passes
+            if (ok) {
+                mbar_expect_tx(smem_u32(&bars.v_full), (uint32_t)kblocks * kTileBytes);
+                for (int kb = 0; kb < kblocks; ++kb)
+                    tma_load_2d(s_kv + kb * kTileBytes, &map_v, 0, bh * a.L + kb * kTile, smem_u32(&bars.v_full));
+                ok = mbar_wait(smem_u32(&bars.v_full), 0, abortp, a.status);
+            }
+            if (ok) ok = mbar_wait(smem_u32(&bars.p_ready), 0, abortp, a.status);
+            // ---- second contraction: O = sum over key blocks, four k-steps of 32 keys each
+            if (ok) {
+                tcgen05_fence_after();
+                for (int kb = 0; kb < kblocks; ++kb) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
+                        const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
+                        tcgen05_mma_i8(tmem + 256, da, db, kIdescPV, (kb | ks) != 0);
+                    }
+                }
+                tcgen05_commit(smem_u32(&bars.o_full));
+            }
+        }
+    } else {
+        // ===================================================== row warps: thread t owns query row q0 + t
+        const int t = tid;                                   // 0..127 = TMEM lane
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const HeadEntry th = a.table[head];
+        const int32_t mult = a.requant_mult[head];
+        // x = floor((acc*mult + 2^(sh-1)) / 2^sh) is the high word of acc * (mult << (32-sh)) + 2^31
+        const int32_t mult_hi = mult << (32 - a.requant_shift);
+        const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
+        uint8_t *row_base = panel + (t >> 3) * 1024 + (t & 7) * 128;
+        const int swz = t & 7;
+        bool ok = true;
+
+        // ---- phase 1: requantise S into the panel, track the row maximum (requantisation is monotone)
+        int xmax = -128;
+        for (int kb = 0; ok && kb < kblocks; ++kb) {
+            const int sb = kb & 1;
+            ok = mbar_wait(smem_u32(&bars.s_full[sb]), (kb >> 1) & 1, abortp, a.status);
+            if (!ok) break;
+            tcgen05_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+                uint32_t acc[32];
+                tmem_ld32(tmem + lane_addr + sb * 128 + j * 32, acc);
+                uint32_t w[8];
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    int32_t x[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
+                        x[e] = min(max(x[e], -128), 127);
+                        if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
+                        xmax = max(xmax, x[e]);
+                    }
+                    w[g] = prmt(prmt((uint32_t)x[0], (uint32_t)x[1], 0x0040u), prmt((uint32_t)x[2], (uint32_t)x[3], 0x0040u),
+                                0x5410u);
+                }
+                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+                *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+            tcgen05_fence_before();
+            mbar_arrive(smem_u32(&bars.s_free[sb]));
+        }
+
+        if (ok) {
+            // ---- phase 2: sum of the closeness values r = max(x + (D - m), 0) (masked keys sit at -128)
+            const int cm = th.D - xmax;
+            const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
+            const int nchunks = kblocks * 8;
+            uint32_t rsum = 0;
+            for (int c = 0; c < nchunks; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(row_base + (c >> 3) * kPanelBlockBytes + (((c & 7) ^ swz) << 4));
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t s2 = 0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    s2 += __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u) + __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                rsum += (s2 & 0xffffu) + (s2 >> 16);
+            }
+            const int masked = kblocks * kTile - nv;                     // keys stored as -128
+            const int rs = (int)rsum - masked * max(cm - 128, 0);
+            const int F = th.B - th.S * th.D;
+            const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
+            const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
+            const uint32_t rp = rho << (1 - a.out_shift);
+            const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+            // ---- phase 3: probabilities, in place
+            for (int c = 0; c < nchunks; ++c) {
+                uint4 *ptr = reinterpret_cast<uint4 *>(row_base + (c >> 3) * kPanelBlockBytes + (((c & 7) ^ swz) << 4));
+                const uint4 v = *ptr;
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t o[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
+                    const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                    uint32_t q;
+                    if (!CLB) {
+                        const uint64_t pe = mad_wide_u32(prmt(ev, 0, 0x2440u), b1, A);
+                        const uint64_t po = mad_wide_u32(prmt(od, 0, 0x2440u), b1, A);
+                        q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                    } else {
+                        const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
+                        const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
+                        const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
+                        const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
+                        q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                    }
+                    if (CAUSAL) {
+                        const int nb = nv - (c * 16 + 4 * k);
+                        q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
+                    }
+                    o[k] = q;
+                }
+                *ptr = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            // the tensor core reads the panel through the async proxy
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(smem_u32(&bars.p_ready));
+
+            // ---- phase 4: O row out of tensor memory, straight to global memory
+            ok = mbar_wait(smem_u32(&bars.o_full), 0, abortp, a.status);
+            if (ok) {
+                tcgen05_fence_after();
+                int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD;
+#pragma unroll 1
+                for (int j = 0; j < 2; ++j) {
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + 256 + j * 32, acc);
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        *reinterpret_cast<uint4 *>(o_row + j * 32 + 4 * g) =
+                            make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
+                }
+                tcgen05_fence_before();
+            }
+        }
+    }
+
+    // ===================================================== common exit: free the tensor memory
+    __syncthreads();
+    if (warp == 4) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows, 64] uint8 tensor, boxes of 128 rows x 64 bytes, 64-byte swizzle.
+bool make_tile_map(CUtensorMap *map, const void *ptr, uint64_t rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD};
+    const cuuint32_t box[2] = {(cuuint32_t)kD, (cuuint32_t)kTile};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool CLB, bool CAUSAL>
+cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const FusedArgs &a,
+                           cudaStream_t st) {
+    const int nblk = a.L / kTile;
+    const size_t smem = 1024 + (size_t)kTileBytes + (size_t)nblk * kTileBytes + (size_t)kTile * a.L;
+    auto kernel = fused_attention_kernel<CLB, CAUSAL>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const unsigned blocks = (unsigned)((int64_t)a.B * a.H * nblk);
+    kernel<<<blocks, kThreads, smem, st>>>(mq, mk, mv, a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool fused_shape_supported(int32_t L, int32_t d) {
+    return d == kD && L >= kTile && L <= kTile * kMaxBlocks && L % kTile == 0;
+}
+
+cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches) {
+    CUtensorMap mq, mk, mv;
+    const uint64_t rows = (uint64_t)a.B * a.H * a.L;
+    if (!make_tile_map(&mq, a.Q, rows) || !make_tile_map(&mk, a.K, rows) || !make_tile_map(&mv, a.V, rows))
+        return cudaErrorInvalidValue;
+    cudaError_t e;
+    const bool clb = (a.flags & HCCS_RECIP_CLB) != 0, causal = (a.flags & HCCS_CAUSAL) != 0;
+    if (!clb && !causal) e = launch_variant<false, false>(mq, mk, mv, a, stream);
+    else if (clb && !causal) e = launch_variant<true, false>(mq, mk, mv, a, stream);
+    else if (!clb && causal) e = launch_variant<false, true>(mq, mk, mv, a, stream);
+    else e = launch_variant<true, true>(mq, mk, mv, a, stream);
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
 }  // namespace hccs

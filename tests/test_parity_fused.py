@@ -1,0 +1,88 @@
+"""GPU parity of hccs_attention_fused (int8 Q.K^T -> requantise -> HCCS -> P.V, int32 out) against
+the oracle's naive triple loops, bit for bit."""
+import numpy as np
+import pytest
+
+from gpu_util import assert_same, oracle_mode
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(hccs, Q, K, V, theta, mult, sh, n_design, flags=0, out_shift=0):
+    import torch
+    ctx = hccs.Context(0)
+    ctx.hccs_params_upload(theta, n_design, out_shift)
+    dQ, dK, dV = (torch.from_numpy(a).cuda() for a in (Q, K, V))
+    O = torch.full(Q.shape, 0x7EADBEEF, dtype=torch.int32, device="cuda")
+    ctx.hccs_attention_fused(dQ, dK, dV, O, mult, sh, flags)
+    torch.cuda.synchronize()
+    assert ctx.hccs_device_status() == 0, "a bounded device-side wait gave up"
+    out = O.cpu().numpy()
+    ctx.close()
+    return out
+
+
+def _rand_qkv(rng, shape, lo=-64, hi=64):
+    return tuple(rng.integers(lo, hi, size=shape, dtype=np.int8) for _ in range(3))
+
+
+@pytest.mark.parametrize("L", [128, 256, 640, 1024])
+@pytest.mark.parametrize("flags", [0, 2, 4, 6])
+def test_small_heads(hccs, oracle, L, flags):
+    rng = np.random.default_rng(1000 + L + flags)
+    Bt, H, d = 1, 3, 64
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d))
+    theta = hccs.workloads.sample_theta(rng, H, L)
+    mult = rng.integers(768, 3841, size=H).astype(np.int32)
+    got = _run(hccs, Q, K, V, theta, mult, 20, L, flags)
+    want = oracle.attention(Q, K, V, mult, 20, theta, oracle_mode(oracle, flags), threads=8)
+    assert_same(got, want, f"fused L={L} flags={flags}")
+
+
+def test_full_range_int8_and_saturating_requant(hccs, oracle):
+    """Operands over all of int8 (|acc| up to 2^20) with multipliers that drive the logits into
+    the int8 clamp; also OUT_SHIFT = 1 and a table designed for more keys than the call uses."""
+    rng = np.random.default_rng(5)
+    Bt, H, L, d = 2, 2, 256, 64
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
+    theta = hccs.workloads.sample_theta(rng, H, 512)
+    mult = np.array([8191, 37], dtype=np.int32)
+    for sh, out_shift in ((20, 0), (16, 1), (31, 0)):
+        if mult.max() >= 2 ** (sh - 1):
+            continue
+        got = _run(hccs, Q, K, V, theta, mult, sh, 512, 0, out_shift)
+        want = oracle.attention(Q, K, V, mult, sh, theta, 0, out_shift, threads=8)
+        assert_same(got, want, f"fused full-range sh={sh} os={out_shift}")
+
+
+def test_config5_sampled_heads(hccs, oracle):
+    """The benchmark's fused workload at full size; the oracle recomputes a sample of heads."""
+    wl = hccs.workloads.make_config(5)
+    got = _run(hccs, wl.Q, wl.K, wl.V, wl.theta, wl.requant_mult, wl.requant_shift, wl.n_design)
+    Bt, H, L, d = wl.shape
+    rng = np.random.default_rng(0)
+    heads = sorted(set(int(v) for v in rng.integers(0, Bt * H, size=10)) | {0, Bt * H - 1})
+    g = got.reshape(Bt * H, L, d)
+    for bh in heads:
+        want = oracle.attention(wl.Q, wl.K, wl.V, wl.requant_mult, wl.requant_shift, wl.theta,
+                                bh_range=(bh, bh + 1), threads=1).reshape(Bt * H, L, d)
+        assert_same(g[bh], want[bh], f"config5 head slice {bh}")
+    assert (got != 0x7EADBEEF).all()
+
+
+def test_unsupported_shapes_are_refused(hccs):
+    import torch
+    ctx = hccs.Context(0)
+    ctx.hccs_params_upload([(31, 1, 20)] * 2, 1024)
+    for L, d in ((100, 64), (128, 32), (2048, 64)):
+        q = torch.zeros((1, 2, L, d), dtype=torch.int8, device="cuda")
+        o = torch.zeros((1, 2, L, d), dtype=torch.int32, device="cuda")
+        with pytest.raises(hccs.HccsError) as ei:
+            ctx.hccs_attention_fused(q, q, q, o, [1000, 1000], 20, 0)
+        assert ei.value.status in (hccs.HCCS_ERR_UNSUPPORTED, hccs.HCCS_ERR_CONSTRAINT)
+    q = torch.zeros((1, 2, 128, 64), dtype=torch.int8, device="cuda")
+    o = torch.zeros((1, 2, 128, 64), dtype=torch.int32, device="cuda")
+    with pytest.raises(hccs.HccsError) as ei:
+        ctx.hccs_attention_fused(q, q, q, o, [1000, 1000], 20, hccs.HCCS_OUT_U16)
+    assert ei.value.status == hccs.HCCS_ERR_UNSUPPORTED
+    ctx.close()
