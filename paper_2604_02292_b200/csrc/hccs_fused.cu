@@ -17,8 +17,10 @@
 //   * V is used as stored ([key][64], keys outermost): that is exactly the MN-major, 64-byte
 //     swizzled B operand, so no transposition is needed.
 //
-// Warp roles (160 threads): warps 0-3 own the 128 rows (TMEM lane quarter = warp index); warp 4
-// lane 0 issues every TMA copy and every MMA.  All mbarrier waits are bounded; a wait that runs
+// Warp roles (288 threads): warps 0-7 are row warps, two threads per query row (thread t and
+// t + 128 both own row t mod 128; TMEM lane quarter = warp index mod 4).  The first of the pair
+// takes the even key blocks, the second the odd ones, and the two exchange their partial row max
+// and row sum through shared memory.  Warp 8 lane 0 issues every TMA copy and every MMA.  All mbarrier waits are bounded; a wait that runs
 // out sets STATUS_FUSED_TIMEOUT, raises an abort flag that every other wait observes, and the CTA
 // leaves through the common exit, which frees its tensor memory.  No clusters, no multicast.
 #include <cuda.h>
@@ -32,8 +34,9 @@ namespace hccs {
 
 namespace {
 
-constexpr int kRowThreads = 128;
-constexpr int kThreads = 160;
+constexpr int kRowThreads = 256;           // two per query row
+constexpr int kThreads = 288;
+constexpr int kCtlWarp = 8;
 constexpr int kD = 64;                    // head dimension (bytes per Q/K/V row)
 constexpr int kTile = 128;                // queries per CTA, keys per block
 constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
@@ -57,6 +60,13 @@ __device__ __forceinline__ uint64_t mad_wide_u32(uint32_t a, uint32_t b, uint64_
 __device__ __forceinline__ int64_t mad_wide_s32(int32_t a, int32_t b, int64_t c) {
     int64_t d;
     asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+// d = { sat8(b), sat8(a), c.lo16 } from low byte up: two signed 32-bit values clamped to int8 and
+// packed below the low half of c.
+__device__ __forceinline__ uint32_t cvt_pack_s8(int32_t a, int32_t b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -159,6 +169,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     __shared__ __align__(8) FusedSmemBarriers bars;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int pair_max[2][kTile], pair_sum[2][kTile];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nblk = a.L / kTile;                         // key blocks (and query tiles) per head
@@ -184,14 +195,14 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         mbar_init(smem_u32(&bars.v_full), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.s_free[i]), kRowThreads);
+            mbar_init(smem_u32(&bars.s_free[i]), kTile);
         }
         mbar_init(smem_u32(&bars.p_ready), kRowThreads);
         mbar_init(smem_u32(&bars.o_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 4) {   // one warp allocates the tensor memory for the CTA
+    if (warp == kCtlWarp) {   // one warp allocates the tensor memory for the CTA
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(kTmemCols)
                      : "memory");
@@ -202,7 +213,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     tcgen05_fence_after();
     const uint32_t tmem = tmem_base_slot;
 
-    if (warp == 4) {
+    if (warp == kCtlWarp) {
         // ===================================================== control thread: TMA + MMA issue
         if (lane == 0) {
             bool ok = true;
@@ -255,9 +266,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             }
         }
     } else {
-        // ===================================================== row warps: thread t owns query row q0 + t
-        const int t = tid;                                   // 0..127 = TMEM lane
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        // ===================================================== row warps: threads t and t + 128 own query row q0 + t
+        const int t = tid & (kTile - 1);                     // TMEM lane = row of the tile
+        const int half = tid >> 7;                           // 0: even key blocks, 1: odd key blocks
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const HeadEntry th = a.table[head];
         const int32_t mult = a.requant_mult[head];
         // x = floor((acc*mult + 2^(sh-1)) / 2^sh) is the high word of acc * (mult << (32-sh)) + 2^31
@@ -269,15 +281,15 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 
         // ---- phase 1: requantise S into the panel, track the row maximum (requantisation is monotone)
         int xmax = -128;
-        for (int kb = 0; ok && kb < kblocks; ++kb) {
-            const int sb = kb & 1;
-            ok = mbar_wait(smem_u32(&bars.s_full[sb]), (kb >> 1) & 1, abortp, a.status);
+        for (int kb = half; ok && kb < kblocks; kb += 2) {
+            ok = mbar_wait(smem_u32(&bars.s_full[half]), (kb >> 1) & 1, abortp, a.status);
             if (!ok) break;
             tcgen05_fence_after();
+            uint8_t *blk = row_base + kb * kPanelBlockBytes;
 #pragma unroll 1
             for (int j = 0; j < 4; ++j) {
                 uint32_t acc[32];
-                tmem_ld32(tmem + lane_addr + sb * 128 + j * 32, acc);
+                tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
                 uint32_t w[8];
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
@@ -285,100 +297,113 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
-                        x[e] = min(max(x[e], -128), 127);
                         if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
-                        xmax = max(xmax, x[e]);
                     }
-                    w[g] = prmt(prmt((uint32_t)x[0], (uint32_t)x[1], 0x0040u), prmt((uint32_t)x[2], (uint32_t)x[3], 0x0040u),
-                                0x5410u);
+                    // two saturating pack steps clamp to int8 and assemble the word
+                    w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
+                    xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
                 }
-                uint8_t *blk = row_base + kb * kPanelBlockBytes;
                 *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
             }
             tcgen05_fence_before();
-            mbar_arrive(smem_u32(&bars.s_free[sb]));
+            mbar_arrive(smem_u32(&bars.s_free[half]));
         }
+        xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
+        pair_max[half][t] = xmax;
+        asm volatile("bar.sync 1, 256;" ::: "memory");        // the row threads only
+        xmax = max(xmax, pair_max[half ^ 1][t]);
 
-        if (ok) {
-            // ---- phase 2: sum of the closeness values r = max(x + (D - m), 0) (masked keys sit at -128)
-            const int cm = th.D - xmax;
-            const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
-            const int nchunks = kblocks * 8;
-            uint32_t rsum = 0;
-            for (int c = 0; c < nchunks; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4 *>(row_base + (c >> 3) * kPanelBlockBytes + (((c & 7) ^ swz) << 4));
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                uint32_t s2 = 0;
+        // ---- phase 2: closeness r = max(x + (D - m), 0), stored back in place of the logit; its sum
+        const int cm = th.D - xmax;
+        const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
+        uint32_t rsum = 0;
+        for (int kb = half; kb < kblocks; kb += 2) {
+            uint8_t *blk = row_base + kb * kPanelBlockBytes;
+            uint4 v[8];
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    s2 += __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u) + __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
-                rsum += (s2 & 0xffffu) + (s2 >> 16);
-            }
-            const int masked = kblocks * kTile - nv;                     // keys stored as -128
-            const int rs = (int)rsum - masked * max(cm - 128, 0);
-            const int F = th.B - th.S * th.D;
-            const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
-            const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
-            const uint32_t rp = rho << (1 - a.out_shift);
-            const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
-            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
-            // ---- phase 3: probabilities, in place
-            for (int c = 0; c < nchunks; ++c) {
-                uint4 *ptr = reinterpret_cast<uint4 *>(row_base + (c >> 3) * kPanelBlockBytes + (((c & 7) ^ swz) << 4));
-                const uint4 v = *ptr;
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                uint32_t o[4];
+            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + ((c ^ swz) << 4));
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                uint32_t s2 = 0;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
                     const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                    s2 += ev + od;
+                    w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
+                }
+                rsum += (s2 & 0xffffu) + (s2 >> 16);
+                *reinterpret_cast<uint4 *>(blk + ((c ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        pair_sum[half][t] = (int)rsum;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const int rs_all = (int)rsum + pair_sum[half ^ 1][t];
+        const int masked = kblocks * kTile - nv;                         // keys stored as -128
+        const int rs = rs_all - masked * max(cm - 128, 0);
+        const int F = th.B - th.S * th.D;
+        const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
+        const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
+        const uint32_t rp = rho << (1 - a.out_shift);
+        const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+        const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+
+        // ---- phase 3: probabilities from the stored closeness values, in place
+        for (int kb = half; kb < kblocks; kb += 2) {
+            uint8_t *blk = row_base + kb * kPanelBlockBytes;
+            uint4 v[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + ((c ^ swz) << 4));
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                uint32_t o[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
                     uint32_t q;
                     if (!CLB) {
-                        const uint64_t pe = mad_wide_u32(prmt(ev, 0, 0x2440u), b1, A);
-                        const uint64_t po = mad_wide_u32(prmt(od, 0, 0x2440u), b1, A);
+                        const uint64_t pe = mad_wide_u32(prmt(w[k], 0, 0x2440u), b1, A);   // keys 0, 2
+                        const uint64_t po = mad_wide_u32(prmt(w[k], 0, 0x3441u), b1, A);   // keys 1, 3
                         q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
                     } else {
-                        const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
-                        const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
-                        const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
-                        const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
+                        const uint32_t x0 = min(a1 + b1 * (w[k] & 0xffu), 0x00ffffffu);
+                        const uint32_t x1 = min(a1 + b1 * prmt(w[k], 0, 0x4441u), 0x00ffffffu);
+                        const uint32_t x2 = min(a1 + b1 * prmt(w[k], 0, 0x4442u), 0x00ffffffu);
+                        const uint32_t x3 = min(a1 + b1 * (w[k] >> 24), 0x00ffffffu);
                         q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
                     }
                     if (CAUSAL) {
-                        const int nb = nv - (c * 16 + 4 * k);
+                        const int nb = nv - (kb * kTile + c * 16 + 4 * k);
                         q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
                     }
                     o[k] = q;
                 }
-                *ptr = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(blk + ((c ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
-            // the tensor core reads the panel through the async proxy
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(smem_u32(&bars.p_ready));
+        }
+        // the tensor core reads the panel through the async proxy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&bars.p_ready));
 
-            // ---- phase 4: O row out of tensor memory, straight to global memory
-            ok = mbar_wait(smem_u32(&bars.o_full), 0, abortp, a.status);
-            if (ok) {
-                tcgen05_fence_after();
-                int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD;
-#pragma unroll 1
-                for (int j = 0; j < 2; ++j) {
-                    uint32_t acc[32];
-                    tmem_ld32(tmem + lane_addr + 256 + j * 32, acc);
+        // ---- phase 4: O row out of tensor memory, straight to global memory (32 columns per thread)
+        if (ok) ok = mbar_wait(smem_u32(&bars.o_full), 0, abortp, a.status);
+        if (ok) {
+            tcgen05_fence_after();
+            int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD + half * 32;
+            uint32_t acc[32];
+            tmem_ld32(tmem + lane_addr + 256 + half * 32, acc);
 #pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        *reinterpret_cast<uint4 *>(o_row + j * 32 + 4 * g) =
-                            make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
-                }
-                tcgen05_fence_before();
-            }
+            for (int g = 0; g < 8; ++g)
+                *reinterpret_cast<uint4 *>(o_row + 4 * g) = make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
+            tcgen05_fence_before();
         }
     }
 
     // ===================================================== common exit: free the tensor memory
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kCtlWarp) {
         tcgen05_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
