@@ -17,10 +17,12 @@
 //   * V is used as stored ([key][64], keys outermost): that is exactly the MN-major, 64-byte
 //     swizzled B operand, so no transposition is needed.
 //
-// Warp roles (288 threads): warps 0-7 are row warps, two threads per query row (thread t and
-// t + 128 both own row t mod 128; TMEM lane quarter = warp index mod 4).  The first of the pair
-// takes the even key blocks, the second the odd ones, and the two exchange their partial row max
-// and row sum through shared memory.  Warp 8 lane 0 issues every TMA copy and every MMA.  All mbarrier waits are bounded; a wait that runs
+// Warp roles (544 threads): warps 0-15 are row warps, four threads per query row (threads t,
+// t + 128, t + 256, t + 384 own row t mod 128; TMEM lane quarter = warp index mod 4): bit 7 of
+// the thread index selects even or odd key blocks, bit 8 the left or right 64 keys of a block.
+// The four exchange their partial row max and row sum through shared memory; the many warps are
+// what hides the latency of the dependent integer chains.  Warp 16 lane 0 issues every TMA copy
+// and every MMA.  All mbarrier waits are bounded; a wait that runs
 // out sets STATUS_FUSED_TIMEOUT, raises an abort flag that every other wait observes, and the CTA
 // leaves through the common exit, which frees its tensor memory.  No clusters, no multicast.
 #include <cuda.h>
@@ -34,9 +36,9 @@ namespace hccs {
 
 namespace {
 
-constexpr int kRowThreads = 256;           // two per query row
-constexpr int kThreads = 288;
-constexpr int kCtlWarp = 8;
+constexpr int kRowThreads = 512;           // four per query row
+constexpr int kThreads = 544;
+constexpr int kCtlWarp = 16;
 constexpr int kD = 64;                    // head dimension (bytes per Q/K/V row)
 constexpr int kTile = 128;                // queries per CTA, keys per block
 constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
@@ -134,6 +136,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor: start address, leading/stride byte offsets (all >> 4), the
 // Blackwell version field (1 at bit 46) and the swizzle mode in bits [61,64).
@@ -169,7 +181,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     __shared__ __align__(8) FusedSmemBarriers bars;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ int pair_max[2][kTile], pair_sum[2][kTile];
+    __shared__ int part_max[4][kTile], part_sum[4][kTile];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nblk = a.L / kTile;                         // key blocks (and query tiles) per head
@@ -195,7 +207,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         mbar_init(smem_u32(&bars.v_full), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.s_free[i]), kTile);
+            mbar_init(smem_u32(&bars.s_free[i]), 2 * kTile);
         }
         mbar_init(smem_u32(&bars.p_ready), kRowThreads);
         mbar_init(smem_u32(&bars.o_full), 1);
@@ -268,51 +280,104 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     } else {
         // ===================================================== row warps: threads t and t + 128 own query row q0 + t
         const int t = tid & (kTile - 1);                     // TMEM lane = row of the tile
-        const int half = tid >> 7;                           // 0: even key blocks, 1: odd key blocks
+        const int grp = tid >> 7;                            // 0..3
+        const int half = grp & 1;                            // 0: even key blocks, 1: odd key blocks
+        const int side = grp >> 1;                           // 0: keys 0-63 of a block, 1: keys 64-127
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const HeadEntry th = a.table[head];
         const int32_t mult = a.requant_mult[head];
-        // x = floor((acc*mult + 2^(sh-1)) / 2^sh) is the high word of acc * (mult << (32-sh)) + 2^31
-        const int32_t mult_hi = mult << (32 - a.requant_shift);
         const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
         uint8_t *row_base = panel + (t >> 3) * 1024 + (t & 7) * 128;
         const int swz = t & 7;
         bool ok = true;
 
-        // ---- phase 1: requantise S into the panel, track the row maximum (requantisation is monotone)
+        // ---- phase 1: requantise S into the panel and track the row maximum.
+        // x = clamp(floor((acc*M + R) / 2^sh), -128, 127) with R = 2^(sh-1).  The map is monotone
+        // and M < 2^(sh-1) makes its steps smaller than one, so clamping acc to [lo, hi] -- the
+        // accumulators that land exactly on -128 and 127 -- gives the same result with no later
+        // clamp.  With y = clamp(acc - lo, 0, hi - lo) (one instruction) and k = 24 - sh,
+        // t = y*(M << k) + ((lo*M + R) << k) lies in [-2^31, 2^31) and x is its top byte: one 32-bit
+        // multiply-add per logit, no shift, and the bytes are picked up by the packing PRMTs.
+        // Shifts above 24 take the 64-bit multiply instead.
         int xmax = -128;
-        for (int kb = half; ok && kb < kblocks; kb += 2) {
-            ok = mbar_wait(smem_u32(&bars.s_full[half]), (kb >> 1) & 1, abortp, a.status);
-            if (!ok) break;
-            tcgen05_fence_after();
-            uint8_t *blk = row_base + kb * kPanelBlockBytes;
-#pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
-                uint32_t acc[32];
-                tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
-                uint32_t w[8];
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    int32_t x[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
-                        if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
-                    }
-                    // two saturating pack steps clamp to int8 and assemble the word
-                    w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
-                    xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
-                }
-                *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        if (a.requant_shift <= 24) {
+            const int sh = a.requant_shift, k = 24 - sh;
+            const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
+            int64_t lo64 = -lim, hi64 = lim;
+            if (mult > 0) {
+                lo64 = -((((int64_t)128 << sh) + R) / mult);
+                hi64 = (((int64_t)128 << sh) - 1 - R) / mult;
+                lo64 = max(lo64, -lim);
+                hi64 = min(hi64, lim);
             }
-            tcgen05_fence_before();
-            mbar_arrive(smem_u32(&bars.s_free[half]));
+            const int neg_lo = (int)-lo64, span = (int)(hi64 - lo64);
+            const uint32_t mk = (uint32_t)mult << k;
+            const uint32_t ck = (uint32_t)(uint64_t)((lo64 * mult + R) * ((int64_t)1 << k));
+            int ymax = 0;
+            for (int kb = half; ok && kb < kblocks; kb += 2) {
+                ok = mbar_wait(smem_u32(&bars.s_full[half]), (kb >> 1) & 1, abortp, a.status);
+                if (!ok) break;
+                tcgen05_fence_after();
+                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+#pragma unroll 1
+                for (int j = 2 * side; j < 2 * side + 2; ++j) {
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
+                    uint32_t w[8];
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        uint32_t tt[4];
+                        int y[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            y[e] = __viaddmin_s32_relu((int)acc[4 * g + e], neg_lo, span);
+                            tt[e] = (uint32_t)y[e] * mk + ck;
+                            if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) { tt[e] = 0x80000000u; y[e] = 0; }
+                        }
+                        w[g] = prmt(prmt(tt[0], tt[1], 0x0073u), prmt(tt[2], tt[3], 0x0073u), 0x5410u);
+                        ymax = __vimax3_s32(__vimax3_s32(ymax, y[0], y[1]), y[2], y[3]);
+                    }
+                    *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+                tcgen05_fence_before();
+                mbar_arrive(smem_u32(&bars.s_free[half]));
+            }
+            xmax = (int)((uint32_t)ymax * mk + ck) >> 24;
+        } else {
+            const int32_t mult_hi = mult << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
+            for (int kb = half; ok && kb < kblocks; kb += 2) {
+                ok = mbar_wait(smem_u32(&bars.s_full[half]), (kb >> 1) & 1, abortp, a.status);
+                if (!ok) break;
+                tcgen05_fence_after();
+                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+#pragma unroll 1
+                for (int j = 2 * side; j < 2 * side + 2; ++j) {
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
+                    uint32_t w[8];
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        int32_t x[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
+                            if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
+                        }
+                        w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
+                        xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
+                    }
+                    *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+                tcgen05_fence_before();
+                mbar_arrive(smem_u32(&bars.s_free[half]));
+            }
         }
         xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
-        pair_max[half][t] = xmax;
-        asm volatile("bar.sync 1, 256;" ::: "memory");        // the row threads only
-        xmax = max(xmax, pair_max[half ^ 1][t]);
+        part_max[grp][t] = xmax;
+        asm volatile("bar.sync 1, 512;" ::: "memory");        // the row threads only
+        xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
 
         // ---- phase 2: closeness r = max(x + (D - m), 0), stored back in place of the logit; its sum
         const int cm = th.D - xmax;
@@ -320,11 +385,11 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         uint32_t rsum = 0;
         for (int kb = half; kb < kblocks; kb += 2) {
             uint8_t *blk = row_base + kb * kPanelBlockBytes;
-            uint4 v[8];
+            uint4 v[4];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + ((c ^ swz) << 4));
+            for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
                 uint32_t s2 = 0;
 #pragma unroll
@@ -335,12 +400,12 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
                 }
                 rsum += (s2 & 0xffffu) + (s2 >> 16);
-                *reinterpret_cast<uint4 *>(blk + ((c ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
-        pair_sum[half][t] = (int)rsum;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        const int rs_all = (int)rsum + pair_sum[half ^ 1][t];
+        part_sum[grp][t] = (int)rsum;
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        const int rs_all = part_sum[0][t] + part_sum[1][t] + part_sum[2][t] + part_sum[3][t];
         const int masked = kblocks * kTile - nv;                         // keys stored as -128
         const int rs = rs_all - masked * max(cm - 128, 0);
         const int F = th.B - th.S * th.D;
@@ -353,11 +418,11 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         // ---- phase 3: probabilities from the stored closeness values, in place
         for (int kb = half; kb < kblocks; kb += 2) {
             uint8_t *blk = row_base + kb * kPanelBlockBytes;
-            uint4 v[8];
+            uint4 v[4];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + ((c ^ swz) << 4));
+            for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
                 uint32_t o[4];
 #pragma unroll
@@ -375,27 +440,27 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
                     }
                     if (CAUSAL) {
-                        const int nb = nv - (kb * kTile + c * 16 + 4 * k);
+                        const int nb = nv - (kb * kTile + (4 * side + c) * 16 + 4 * k);
                         q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
                     }
                     o[k] = q;
                 }
-                *reinterpret_cast<uint4 *>(blk + ((c ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
         // the tensor core reads the panel through the async proxy
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(smem_u32(&bars.p_ready));
 
-        // ---- phase 4: O row out of tensor memory, straight to global memory (32 columns per thread)
+        // ---- phase 4: O row out of tensor memory, straight to global memory (16 columns per thread)
         if (ok) ok = mbar_wait(smem_u32(&bars.o_full), 0, abortp, a.status);
         if (ok) {
             tcgen05_fence_after();
-            int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD + half * 32;
-            uint32_t acc[32];
-            tmem_ld32(tmem + lane_addr + 256 + half * 32, acc);
+            int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD + grp * 16;
+            uint32_t acc[16];
+            tmem_ld16(tmem + lane_addr + 256 + grp * 16, acc);
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
+            for (int g = 0; g < 4; ++g)
                 *reinterpret_cast<uint4 *>(o_row + 4 * g) = make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
             tcgen05_fence_before();
         }

@@ -6,7 +6,7 @@
 // instructions.  Each 32-bit word of four int8 logits is therefore split once into two words of
 // two sign-extended 16-bit lanes (bytes 0,2 and bytes 1,3; one PRMT each), and every later stage
 // works on those:
-//   stage 1  m = max x                      one max.s16x2 per split word
+//   stage 1  m = max x                      one three-input max.s16x2 per word
 //   stage 2+3  instead of delta = min(m - x, D) the kernel keeps the "closeness"
 //            r = D - delta = max(x + (D - m), 0)   one viaddmax.s16x2 per split word
 //            so that the score is s = B - S*delta = F + S*r with F = B - S*D (Eq. 2, Eq. 3);
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
             const uint32_t ev = prmt(w, 0, kSelEven), od = prmt(w, 0, kSelOdd);
             e[8 * v + k] = ev;
             o[8 * v + k] = od;
-            M = __vmaxs2(M, __vmaxs2(ev, od));
+            M = __vimax3_s16x2(M, ev, od);
         }
     }
     int m = max((int)(short)(M & 0xffffu), (int)M >> 16);
