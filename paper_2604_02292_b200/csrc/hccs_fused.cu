@@ -169,7 +169,7 @@ struct FusedSmemBarriers {
     uint64_t v_full;
     uint64_t s_full[2];
     uint64_t s_free[2];
-    uint64_t p_ready;
+    uint64_t p_ready[kMaxBlocks];   // block kb of the probability panel is complete
     uint64_t o_full;
 };
 
@@ -209,7 +209,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             mbar_init(smem_u32(&bars.s_full[i]), 1);
             mbar_init(smem_u32(&bars.s_free[i]), 2 * kTile);
         }
-        mbar_init(smem_u32(&bars.p_ready), kRowThreads);
+        for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.p_ready[i]), kRowThreads / 2);
         mbar_init(smem_u32(&bars.o_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -262,18 +262,20 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     tma_load_2d(s_kv + kb * kTileBytes, &map_v, 0, bh * a.L + kb * kTile, smem_u32(&bars.v_full));
                 ok = mbar_wait(smem_u32(&bars.v_full), 0, abortp, a.status);
             }
-            if (ok) ok = mbar_wait(smem_u32(&bars.p_ready), 0, abortp, a.status);
-            // ---- second contraction: O = sum over key blocks, four k-steps of 32 keys each
-            if (ok) {
+            // ---- second contraction, block by block as the row warps finish the probabilities:
+            // four k-steps of 32 keys per block
+            for (int kb = 0; ok && kb < kblocks; ++kb) {
+                ok = mbar_wait(smem_u32(&bars.p_ready[kb]), 0, abortp, a.status);
+                if (!ok) break;
                 tcgen05_fence_after();
-                for (int kb = 0; kb < kblocks; ++kb) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
-                        const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
-                        tcgen05_mma_i8(tmem + 256, da, db, kIdescPV, (kb | ks) != 0);
-                    }
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
+                    const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
+                    tcgen05_mma_i8(tmem + 256, da, db, kIdescPV, (kb | ks) != 0);
                 }
+            }
+            if (ok) {
                 tcgen05_commit(smem_u32(&bars.o_full));
             }
         }
@@ -447,22 +449,36 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 }
                 *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
+            // the tensor core reads the panel through the async proxy: hand this block over
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(smem_u32(&bars.p_ready[kb]));
         }
-        // the tensor core reads the panel through the async proxy
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(smem_u32(&bars.p_ready));
 
-        // ---- phase 4: O row out of tensor memory, straight to global memory (16 columns per thread)
+        // ---- phase 4: O out of tensor memory.  A thread holds 16 columns of its row; writing them
+        // straight to global memory would cost one memory transaction per lane (rows are 256 bytes
+        // apart), so the tile goes through shared memory (K/V buffer, free now; rows padded to 272
+        // bytes to spread the banks) and leaves as one 256-byte bulk copy per row.
         if (ok) ok = mbar_wait(smem_u32(&bars.o_full), 0, abortp, a.status);
+        uint8_t *o_stage = gen_base + kTileBytes + t * 272;
         if (ok) {
             tcgen05_fence_after();
-            int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD + grp * 16;
             uint32_t acc[16];
             tmem_ld16(tmem + lane_addr + 256 + grp * 16, acc);
 #pragma unroll
             for (int g = 0; g < 4; ++g)
-                *reinterpret_cast<uint4 *>(o_row + 4 * g) = make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
+                *reinterpret_cast<uint4 *>(o_stage + grp * 64 + g * 16) =
+                    make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
             tcgen05_fence_before();
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        if (ok && grp == 0) {
+            int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(o_row),
+                         "r"(s_kv + t * 272)
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem must outlive the read
         }
     }
 
@@ -508,7 +524,9 @@ template <bool CLB, bool CAUSAL>
 cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const FusedArgs &a,
                            cudaStream_t st) {
     const int nblk = a.L / kTile;
-    const size_t smem = 1024 + (size_t)kTileBytes + (size_t)nblk * kTileBytes + (size_t)kTile * a.L;
+    size_t work = (size_t)nblk * kTileBytes + (size_t)kTile * a.L;   // K/V tiles + panel
+    if (work < (size_t)kTile * 272) work = (size_t)kTile * 272;       // the O staging rows reuse that space
+    const size_t smem = 1024 + (size_t)kTileBytes + work;
     auto kernel = fused_attention_kernel<CLB, CAUSAL>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
