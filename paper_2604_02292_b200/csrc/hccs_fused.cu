@@ -176,28 +176,26 @@ struct FusedSmemBarriers {
 template <bool CLB, bool CAUSAL>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                       const __grid_constant__ CUtensorMap map_v, FusedArgs a) {
+                       const __grid_constant__ CUtensorMap map_v, FusedArgs a, int num_tiles) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) FusedSmemBarriers bars;
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ int abort_flag, leave_flag;
     __shared__ int part_max[4][kTile], part_sum[4][kTile];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nblk = a.L / kTile;                         // key blocks (and query tiles) per head
-    const int bh = blockIdx.x / nblk, qt = blockIdx.x % nblk;
-    const int head = bh % a.H;
-    const int q0 = qt * kTile;
-    const int kblocks = CAUSAL ? qt + 1 : nblk;           // key blocks this tile needs
     volatile int *abortp = &abort_flag;
 
     // shared-memory carve-up (1024-byte aligned: required by the swizzled layouts)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_q = base;                                            // Q tile
-    const uint32_t s_kv = base + kTileBytes;                              // K tiles, later V tiles
+    const uint32_t s_kpre = s_q + kTileBytes;                             // K blocks 0 and 1 (prefetched)
+    const uint32_t s_kv = s_kpre + 2 * kTileBytes;                        // K blocks 2.., later all V blocks
     const uint32_t s_p = s_kv + (uint32_t)nblk * kTileBytes;              // logit / probability panel
-    uint8_t *panel = gen_base + kTileBytes + (size_t)nblk * kTileBytes;
+    uint8_t *panel = gen_base + 3 * kTileBytes + (size_t)nblk * kTileBytes;
+    auto k_slot = [&](int kb) { return kb < 2 ? s_kpre + kb * kTileBytes : s_kv + kb * kTileBytes; };
 
     if (tid == 0) {
         abort_flag = 0;
@@ -225,261 +223,310 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     tcgen05_fence_after();
     const uint32_t tmem = tmem_base_slot;
 
+    // A CTA walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every mbarrier completes
+    // one phase per use, so both sides count their uses (per barrier, because a causal tile uses
+    // only its first qt + 1 key blocks) and wait on the parity of that count.
     if (warp == kCtlWarp) {
         // ===================================================== control thread: TMA + MMA issue
         if (lane == 0) {
             bool ok = true;
-            mbar_expect_tx(smem_u32(&bars.q_full), kTileBytes);
-            tma_load_2d(s_q, &map_q, 0, bh * a.L + q0, smem_u32(&bars.q_full));
-            for (int kb = 0; kb < kblocks; ++kb) {
-                mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
-                tma_load_2d(s_kv + kb * kTileBytes, &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
-            }
-            ok = mbar_wait(smem_u32(&bars.q_full), 0, abortp, a.status);
-            // ---- first contraction: S_kb = Q . K_kb^T, two k-steps of 32 over d = 64
-            for (int kb = 0; ok && kb < kblocks; ++kb) {
+            uint32_t q_uses = 0, kdone_uses = 0, v_uses = 0, o_uses = 0;
+            uint32_t k_par = 0, p_par = 0;               // bit kb = parity of the next use of k_full[kb] / p_ready[kb]
+            uint32_t s_uses[2] = {0, 0};
+            // Q and the first two K blocks of a tile go to buffers of their own, so they can be
+            // fetched while the previous tile is still in its softmax passes.
+            auto prefetch = [&](int tile) {
+                const int bh = tile / nblk, qt = tile % nblk;
+                const int kblocks = CAUSAL ? qt + 1 : nblk;
+                mbar_expect_tx(smem_u32(&bars.q_full), kTileBytes);
+                tma_load_2d(s_q, &map_q, 0, bh * a.L + qt * kTile, smem_u32(&bars.q_full));
+                for (int kb = 0; kb < min(2, kblocks); ++kb) {
+                    mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
+                    tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
+                }
+            };
+            auto mma_qk = [&](int kb) {                  // S[kb & 1] = Q . K_kb^T, two k-steps of 32 over d = 64
                 const int sb = kb & 1;
-                if (kb >= 2) ok = mbar_wait(smem_u32(&bars.s_free[sb]), ((kb >> 1) - 1) & 1, abortp, a.status);
-                if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), 0, abortp, a.status);
-                if (!ok) break;
+                if (s_uses[sb] > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (s_uses[sb] - 1) & 1, abortp, a.status);
+                if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
+                if (!ok) return;
+                k_par ^= 1u << kb;
+                ++s_uses[sb];
                 tcgen05_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 2; ++ks) {
                     const uint64_t da = smem_desc(s_q + ks * 32, 16, 512, kSwizzle64);
-                    const uint64_t db = smem_desc(s_kv + kb * kTileBytes + ks * 32, 16, 512, kSwizzle64);
+                    const uint64_t db = smem_desc(k_slot(kb) + ks * 32, 16, 512, kSwizzle64);
                     tcgen05_mma_i8(tmem + sb * 128, da, db, kIdescQK, ks);
                 }
                 tcgen05_commit(smem_u32(&bars.s_full[sb]));
-            }
-            if (ok) {
+            };
+            if ((int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
+            for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                const int bh = tile / nblk, qt = tile % nblk;
+                const int kblocks = CAUSAL ? qt + 1 : nblk;
+                ok = mbar_wait(smem_u32(&bars.q_full), q_uses++ & 1, abortp, a.status);
+                for (int kb = 0; ok && kb < min(2, kblocks); ++kb) mma_qk(kb);
+                // the other K blocks land where the previous tile's V sits: wait for its last MMA
+                if (ok && it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (o_uses - 1) & 1, abortp, a.status);
+                if (!ok) break;
+                for (int kb = 2; kb < kblocks; ++kb) {
+                    mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
+                    tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
+                }
+                for (int kb = 2; ok && kb < kblocks; ++kb) mma_qk(kb);
+                if (!ok) break;
                 tcgen05_commit(smem_u32(&bars.k_done));
-                ok = mbar_wait(smem_u32(&bars.k_done), 0, abortp, a.status);
-            }
-            // ---- V replaces K in shared memory while the row warps run the softmax passes
-            if (ok) {
+                ok = mbar_wait(smem_u32(&bars.k_done), kdone_uses++ & 1, abortp, a.status);
+                if (!ok) break;
+                // ---- V takes the K buffer while the row warps run the softmax passes; Q and the
+                // first K blocks of the next tile are fetched as well
                 mbar_expect_tx(smem_u32(&bars.v_full), (uint32_t)kblocks * kTileBytes);
                 for (int kb = 0; kb < kblocks; ++kb)
                     tma_load_2d(s_kv + kb * kTileBytes, &map_v, 0, bh * a.L + kb * kTile, smem_u32(&bars.v_full));
-                ok = mbar_wait(smem_u32(&bars.v_full), 0, abortp, a.status);
-            }
-            // ---- second contraction, block by block as the row warps finish the probabilities:
-            // four k-steps of 32 keys per block
-            for (int kb = 0; ok && kb < kblocks; ++kb) {
-                ok = mbar_wait(smem_u32(&bars.p_ready[kb]), 0, abortp, a.status);
-                if (!ok) break;
-                tcgen05_fence_after();
+                if (tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
+                ok = mbar_wait(smem_u32(&bars.v_full), v_uses++ & 1, abortp, a.status);
+                // ---- second contraction, block by block as the row warps finish the probabilities:
+                // four k-steps of 32 keys per block
+                for (int kb = 0; ok && kb < kblocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&bars.p_ready[kb]), (p_par >> kb) & 1, abortp, a.status);
+                    if (!ok) break;
+                    p_par ^= 1u << kb;
+                    tcgen05_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
-                    const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
-                    tcgen05_mma_i8(tmem + 256, da, db, kIdescPV, (kb | ks) != 0);
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
+                        const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
+                        tcgen05_mma_i8(tmem + 256, da, db, kIdescPV, (kb | ks) != 0);
+                    }
                 }
-            }
-            if (ok) {
+                if (!ok) break;
                 tcgen05_commit(smem_u32(&bars.o_full));
+                ++o_uses;
             }
         }
     } else {
-        // ===================================================== row warps: threads t and t + 128 own query row q0 + t
+        // ===================================================== row warps: threads t, t+128, t+256, t+384 own query row t
         const int t = tid & (kTile - 1);                     // TMEM lane = row of the tile
         const int grp = tid >> 7;                            // 0..3
         const int half = grp & 1;                            // 0: even key blocks, 1: odd key blocks
         const int side = grp >> 1;                           // 0: keys 0-63 of a block, 1: keys 64-127
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const HeadEntry th = a.table[head];
-        const int32_t mult = a.requant_mult[head];
-        const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
         uint8_t *row_base = panel + (t >> 3) * 1024 + (t & 7) * 128;
         const int swz = t & 7;
+        uint32_t sfull_uses = 0;                             // uses of s_full[half] by this thread
         bool ok = true;
 
-        // ---- phase 1: requantise S into the panel and track the row maximum.
-        // x = clamp(floor((acc*M + R) / 2^sh), -128, 127) with R = 2^(sh-1).  The map is monotone
-        // and M < 2^(sh-1) makes its steps smaller than one, so clamping acc to [lo, hi] -- the
-        // accumulators that land exactly on -128 and 127 -- gives the same result with no later
-        // clamp.  With y = clamp(acc - lo, 0, hi - lo) (one instruction) and k = 24 - sh,
-        // t = y*(M << k) + ((lo*M + R) << k) lies in [-2^31, 2^31) and x is its top byte: one 32-bit
-        // multiply-add per logit, no shift, and the bytes are picked up by the packing PRMTs.
-        // Shifts above 24 take the 64-bit multiply instead.
-        int xmax = -128;
-        if (a.requant_shift <= 24) {
-            const int sh = a.requant_shift, k = 24 - sh;
-            const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
-            int64_t lo64 = -lim, hi64 = lim;
-            if (mult > 0) {
-                lo64 = -((((int64_t)128 << sh) + R) / mult);
-                hi64 = (((int64_t)128 << sh) - 1 - R) / mult;
-                lo64 = max(lo64, -lim);
-                hi64 = min(hi64, lim);
+        for (int tile = blockIdx.x, it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
+            const int bh = tile / nblk, qt = tile % nblk;
+            const int head = bh % a.H;
+            const int q0 = qt * kTile;
+            const int kblocks = CAUSAL ? qt + 1 : nblk;
+            const HeadEntry th = a.table[head];
+            const int32_t mult = a.requant_mult[head];
+            const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
+
+            // the previous tile's O rows were staged in the panel: their bulk copies must have
+            // read them before the panel is written again
+            if (it > 0) {
+                if (grp == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                asm volatile("bar.sync 1, 512;" ::: "memory");
             }
-            const int neg_lo = (int)-lo64, span = (int)(hi64 - lo64);
-            const uint32_t mk = (uint32_t)mult << k;
-            const uint32_t ck = (uint32_t)(uint64_t)((lo64 * mult + R) * ((int64_t)1 << k));
-            int ymax = 0;
-            for (int kb = half; ok && kb < kblocks; kb += 2) {
-                ok = mbar_wait(smem_u32(&bars.s_full[half]), (kb >> 1) & 1, abortp, a.status);
-                if (!ok) break;
-                tcgen05_fence_after();
-                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+
+            // ---- phase 1: requantise S into the panel and track the row maximum.
+            // x = clamp(floor((acc*M + R) / 2^sh), -128, 127) with R = 2^(sh-1).  The map is monotone
+            // and M < 2^(sh-1) makes its steps smaller than one, so clamping acc to [lo, hi] -- the
+            // accumulators that land exactly on -128 and 127 -- gives the same result with no later
+            // clamp.  With y = clamp(acc - lo, 0, hi - lo) (one instruction) and k = 24 - sh,
+            // t = y*(M << k) + ((lo*M + R) << k) lies in [-2^31, 2^31) and x is its top byte: one 32-bit
+            // multiply-add per logit, no shift, and the bytes are picked up by the packing PRMTs.
+            // Shifts above 24 take the 64-bit multiply instead.
+            int xmax = -128;
+            if (a.requant_shift <= 24) {
+                const int sh = a.requant_shift, k = 24 - sh;
+                const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
+                int64_t lo64 = -lim, hi64 = lim;
+                if (mult > 0) {
+                    lo64 = -((((int64_t)128 << sh) + R) / mult);
+                    hi64 = (((int64_t)128 << sh) - 1 - R) / mult;
+                    lo64 = max(lo64, -lim);
+                    hi64 = min(hi64, lim);
+                }
+                const int neg_lo = (int)-lo64, span = (int)(hi64 - lo64);
+                const uint32_t mk = (uint32_t)mult << k;
+                const uint32_t ck = (uint32_t)(uint64_t)((lo64 * mult + R) * ((int64_t)1 << k));
+                int ymax = 0;
+                for (int kb = half; ok && kb < kblocks; kb += 2) {
+                    ok = mbar_wait(smem_u32(&bars.s_full[half]), sfull_uses & 1, abortp, a.status);
+                    if (!ok) break;
+                    ++sfull_uses;
+                    tcgen05_fence_after();
+                    uint8_t *blk = row_base + kb * kPanelBlockBytes;
 #pragma unroll 1
-                for (int j = 2 * side; j < 2 * side + 2; ++j) {
-                    uint32_t acc[32];
-                    tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
-                    uint32_t w[8];
+                    for (int j = 2 * side; j < 2 * side + 2; ++j) {
+                        uint32_t acc[32];
+                        tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
+                        uint32_t w[8];
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        uint32_t tt[4];
-                        int y[4];
+                        for (int g = 0; g < 8; ++g) {
+                            uint32_t tt[4];
+                            int y[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            y[e] = __viaddmin_s32_relu((int)acc[4 * g + e], neg_lo, span);
-                            tt[e] = (uint32_t)y[e] * mk + ck;
-                            if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) { tt[e] = 0x80000000u; y[e] = 0; }
+                            for (int e = 0; e < 4; ++e) {
+                                y[e] = __viaddmin_s32_relu((int)acc[4 * g + e], neg_lo, span);
+                                tt[e] = (uint32_t)y[e] * mk + ck;
+                                if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) { tt[e] = 0x80000000u; y[e] = 0; }
+                            }
+                            w[g] = prmt(prmt(tt[0], tt[1], 0x0073u), prmt(tt[2], tt[3], 0x0073u), 0x5410u);
+                            ymax = __vimax3_s32(__vimax3_s32(ymax, y[0], y[1]), y[2], y[3]);
                         }
-                        w[g] = prmt(prmt(tt[0], tt[1], 0x0073u), prmt(tt[2], tt[3], 0x0073u), 0x5410u);
-                        ymax = __vimax3_s32(__vimax3_s32(ymax, y[0], y[1]), y[2], y[3]);
+                        *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
                     }
-                    *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                    tcgen05_fence_before();
+                    mbar_arrive(smem_u32(&bars.s_free[half]));
                 }
-                tcgen05_fence_before();
-                mbar_arrive(smem_u32(&bars.s_free[half]));
-            }
-            xmax = (int)((uint32_t)ymax * mk + ck) >> 24;
-        } else {
-            const int32_t mult_hi = mult << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
-            for (int kb = half; ok && kb < kblocks; kb += 2) {
-                ok = mbar_wait(smem_u32(&bars.s_full[half]), (kb >> 1) & 1, abortp, a.status);
-                if (!ok) break;
-                tcgen05_fence_after();
-                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+                xmax = (int)((uint32_t)ymax * mk + ck) >> 24;
+            } else {
+                const int32_t mult_hi = mult << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
+                for (int kb = half; ok && kb < kblocks; kb += 2) {
+                    ok = mbar_wait(smem_u32(&bars.s_full[half]), sfull_uses & 1, abortp, a.status);
+                    if (!ok) break;
+                    ++sfull_uses;
+                    tcgen05_fence_after();
+                    uint8_t *blk = row_base + kb * kPanelBlockBytes;
 #pragma unroll 1
-                for (int j = 2 * side; j < 2 * side + 2; ++j) {
-                    uint32_t acc[32];
-                    tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
-                    uint32_t w[8];
+                    for (int j = 2 * side; j < 2 * side + 2; ++j) {
+                        uint32_t acc[32];
+                        tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
+                        uint32_t w[8];
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        int32_t x[4];
+                        for (int g = 0; g < 8; ++g) {
+                            int32_t x[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
-                            if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
+                            for (int e = 0; e < 4; ++e) {
+                                x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
+                                if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
+                            }
+                            w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
+                            xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
                         }
-                        w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
-                        xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
+                        *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
                     }
-                    *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                    tcgen05_fence_before();
+                    mbar_arrive(smem_u32(&bars.s_free[half]));
                 }
+            }
+            xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
+            part_max[grp][t] = xmax;
+            asm volatile("bar.sync 1, 512;" ::: "memory");        // the row threads only
+            xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
+
+            // ---- phase 2: closeness r = max(x + (D - m), 0), stored back in place of the logit; its sum
+            const int cm = th.D - xmax;
+            const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
+            uint32_t rsum = 0;
+            for (int kb = half; kb < kblocks; kb += 2) {
+                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+                uint4 v[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                    uint32_t s2 = 0;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
+                        const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                        s2 += ev + od;
+                        w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
+                    }
+                    rsum += (s2 & 0xffffu) + (s2 >> 16);
+                    *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            part_sum[grp][t] = (int)rsum;
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            const int rs_all = part_sum[0][t] + part_sum[1][t] + part_sum[2][t] + part_sum[3][t];
+            const int masked = kblocks * kTile - nv;                         // keys stored as -128
+            const int rs = rs_all - masked * max(cm - 128, 0);
+            const int F = th.B - th.S * th.D;
+            const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
+            const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
+            const uint32_t rp = rho << (1 - a.out_shift);
+            const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+
+            // ---- phase 3: probabilities from the stored closeness values, in place
+            for (int kb = half; kb < kblocks; kb += 2) {
+                uint8_t *blk = row_base + kb * kPanelBlockBytes;
+                uint4 v[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        uint32_t q;
+                        if (!CLB) {
+                            const uint64_t pe = mad_wide_u32(prmt(w[k], 0, 0x2440u), b1, A);   // keys 0, 2
+                            const uint64_t po = mad_wide_u32(prmt(w[k], 0, 0x3441u), b1, A);   // keys 1, 3
+                            q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                        } else {
+                            const uint32_t x0 = min(a1 + b1 * (w[k] & 0xffu), 0x00ffffffu);
+                            const uint32_t x1 = min(a1 + b1 * prmt(w[k], 0, 0x4441u), 0x00ffffffu);
+                            const uint32_t x2 = min(a1 + b1 * prmt(w[k], 0, 0x4442u), 0x00ffffffu);
+                            const uint32_t x3 = min(a1 + b1 * (w[k] >> 24), 0x00ffffffu);
+                            q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                        }
+                        if (CAUSAL) {
+                            const int nb = nv - (kb * kTile + (4 * side + c) * 16 + 4 * k);
+                            q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
+                        }
+                        o[k] = q;
+                    }
+                    *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+                // the tensor core reads the panel through the async proxy: hand this block over
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(smem_u32(&bars.p_ready[kb]));
+            }
+
+            // ---- phase 4: O out of tensor memory.  A thread holds 16 columns of its row; writing them
+            // straight to global memory would cost one memory transaction per lane (rows are 256 bytes
+            // apart), so the tile goes through shared memory (the panel, free once the second
+            // contraction is complete; rows padded to 272 bytes to spread the banks) and leaves as one
+            // 256-byte bulk copy per row.
+            if (ok) ok = mbar_wait(smem_u32(&bars.o_full), it & 1, abortp, a.status);
+            if (ok) {
+                tcgen05_fence_after();
+                uint32_t acc[16];
+                tmem_ld16(tmem + lane_addr + 256 + grp * 16, acc);
+                uint8_t *o_stage = panel + t * 272;
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    *reinterpret_cast<uint4 *>(o_stage + grp * 64 + g * 16) =
+                        make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
                 tcgen05_fence_before();
-                mbar_arrive(smem_u32(&bars.s_free[half]));
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
-        }
-        xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
-        part_max[grp][t] = xmax;
-        asm volatile("bar.sync 1, 512;" ::: "memory");        // the row threads only
-        xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
-
-        // ---- phase 2: closeness r = max(x + (D - m), 0), stored back in place of the logit; its sum
-        const int cm = th.D - xmax;
-        const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
-        uint32_t rsum = 0;
-        for (int kb = half; kb < kblocks; kb += 2) {
-            uint8_t *blk = row_base + kb * kPanelBlockBytes;
-            uint4 v[4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-                uint32_t s2 = 0;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
-                    const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
-                    s2 += ev + od;
-                    w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
-                }
-                rsum += (s2 & 0xffffu) + (s2 >> 16);
-                *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            if (tid == 0) leave_flag = *abortp;                   // one reader, so that all row threads agree
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (ok && grp == 0) {
+                int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD;
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(o_row),
+                             "r"(s_p + t * 272)
+                             : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
+            // leave the loop together (the flag was sampled once, before the barrier above)
+            if (*(volatile int *)&leave_flag) break;
         }
-        part_sum[grp][t] = (int)rsum;
-        asm volatile("bar.sync 1, 512;" ::: "memory");
-        const int rs_all = part_sum[0][t] + part_sum[1][t] + part_sum[2][t] + part_sum[3][t];
-        const int masked = kblocks * kTile - nv;                         // keys stored as -128
-        const int rs = rs_all - masked * max(cm - 128, 0);
-        const int F = th.B - th.S * th.D;
-        const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
-        const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
-        const uint32_t rp = rho << (1 - a.out_shift);
-        const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
-        const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
-
-        // ---- phase 3: probabilities from the stored closeness values, in place
-        for (int kb = half; kb < kblocks; kb += 2) {
-            uint8_t *blk = row_base + kb * kPanelBlockBytes;
-            uint4 v[4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-                uint32_t o[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    uint32_t q;
-                    if (!CLB) {
-                        const uint64_t pe = mad_wide_u32(prmt(w[k], 0, 0x2440u), b1, A);   // keys 0, 2
-                        const uint64_t po = mad_wide_u32(prmt(w[k], 0, 0x3441u), b1, A);   // keys 1, 3
-                        q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
-                    } else {
-                        const uint32_t x0 = min(a1 + b1 * (w[k] & 0xffu), 0x00ffffffu);
-                        const uint32_t x1 = min(a1 + b1 * prmt(w[k], 0, 0x4441u), 0x00ffffffu);
-                        const uint32_t x2 = min(a1 + b1 * prmt(w[k], 0, 0x4442u), 0x00ffffffu);
-                        const uint32_t x3 = min(a1 + b1 * (w[k] >> 24), 0x00ffffffu);
-                        q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
-                    }
-                    if (CAUSAL) {
-                        const int nb = nv - (kb * kTile + (4 * side + c) * 16 + 4 * k);
-                        q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
-                    }
-                    o[k] = q;
-                }
-                *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-            }
-            // the tensor core reads the panel through the async proxy: hand this block over
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(smem_u32(&bars.p_ready[kb]));
-        }
-
-        // ---- phase 4: O out of tensor memory.  A thread holds 16 columns of its row; writing them
-        // straight to global memory would cost one memory transaction per lane (rows are 256 bytes
-        // apart), so the tile goes through shared memory (K/V buffer, free now; rows padded to 272
-        // bytes to spread the banks) and leaves as one 256-byte bulk copy per row.
-        if (ok) ok = mbar_wait(smem_u32(&bars.o_full), 0, abortp, a.status);
-        uint8_t *o_stage = gen_base + kTileBytes + t * 272;
-        if (ok) {
-            tcgen05_fence_after();
-            uint32_t acc[16];
-            tmem_ld16(tmem + lane_addr + 256 + grp * 16, acc);
-#pragma unroll
-            for (int g = 0; g < 4; ++g)
-                *reinterpret_cast<uint4 *>(o_stage + grp * 64 + g * 16) =
-                    make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
-            tcgen05_fence_before();
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        }
-        asm volatile("bar.sync 1, 512;" ::: "memory");
-        if (ok && grp == 0) {
-            int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD;
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(o_row),
-                         "r"(s_kv + t * 272)
-                         : "memory");
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem must outlive the read
-        }
+        if (grp == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem must outlive the reads
     }
 
     // ===================================================== common exit: free the tensor memory
@@ -524,14 +571,18 @@ template <bool CLB, bool CAUSAL>
 cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const FusedArgs &a,
                            cudaStream_t st) {
     const int nblk = a.L / kTile;
-    size_t work = (size_t)nblk * kTileBytes + (size_t)kTile * a.L;   // K/V tiles + panel
-    if (work < (size_t)kTile * 272) work = (size_t)kTile * 272;       // the O staging rows reuse that space
-    const size_t smem = 1024 + (size_t)kTileBytes + work;
+    size_t panel = (size_t)kTile * a.L;
+    if (panel < (size_t)kTile * 272) panel = (size_t)kTile * 272;     // the O staging rows reuse the panel
+    const size_t smem = 1024 + 3 * (size_t)kTileBytes + (size_t)nblk * kTileBytes + panel;
     auto kernel = fused_attention_kernel<CLB, CAUSAL>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned blocks = (unsigned)((int64_t)a.B * a.H * nblk);
-    kernel<<<blocks, kThreads, smem, st>>>(mq, mk, mv, a);
+    const int64_t tiles = (int64_t)a.B * a.H * nblk;
+    int sms = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const unsigned blocks = (unsigned)(tiles < sms ? tiles : sms);      // persistent: one CTA per SM
+    kernel<<<blocks, kThreads, smem, st>>>(mq, mk, mv, a, (int)tiles);
     return cudaGetLastError();
 }
 
