@@ -18,8 +18,9 @@
 //     swizzled B operand, so no transposition is needed.
 //
 // Warp roles (544 threads): warps 0-15 are row warps, four threads per query row (threads t,
-// t + 128, t + 256, t + 384 own row t mod 128; TMEM lane quarter = warp index mod 4): bit 7 of
-// the thread index selects even or odd key blocks, bit 8 the left or right 64 keys of a block.
+// t + 128, t + 256, t + 384 own row t mod 128; TMEM lane quarter = warp index mod 4): bits 7-8
+// of the thread index select which 32 of the 128 keys of every block the thread handles, so all
+// row threads work on the same block while the tensor core fills the other S buffer.
 // The four exchange their partial row max and row sum through shared memory; the many warps are
 // what hides the latency of the dependent integer chains.  Warp 16 lane 0 issues every TMA copy
 // and every MMA.  All mbarrier waits are bounded; a wait that runs
@@ -83,8 +84,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Bounded, abort-aware wait.  Returns false when the wait was given up (here or elsewhere).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           uint32_t *status) {
-    const long long t0 = clock64();
-    for (;;) {
+    long long t0 = 0;
+    for (uint32_t polls = 0;; ++polls) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -94,8 +95,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             : "r"(bar), "r"(parity)
             : "memory");
         if (done) return true;
+        if ((polls & 31u) != 31u) continue;          // look at the flag and the clock now and then
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        if (now - t0 > kWaitCycles) {
             *abort_flag = 1;
             atomicOr(status, STATUS_FUSED_TIMEOUT);
             return false;
@@ -205,9 +209,9 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         mbar_init(smem_u32(&bars.v_full), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.s_free[i]), 2 * kTile);
+            mbar_init(smem_u32(&bars.s_free[i]), kRowThreads);
         }
-        for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.p_ready[i]), kRowThreads / 2);
+        for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.p_ready[i]), kRowThreads);
         mbar_init(smem_u32(&bars.o_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -308,13 +312,11 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     } else {
         // ===================================================== row warps: threads t, t+128, t+256, t+384 own query row t
         const int t = tid & (kTile - 1);                     // TMEM lane = row of the tile
-        const int grp = tid >> 7;                            // 0..3
-        const int half = grp & 1;                            // 0: even key blocks, 1: odd key blocks
-        const int side = grp >> 1;                           // 0: keys 0-63 of a block, 1: keys 64-127
+        const int grp = tid >> 7;                            // 0..3: keys 32*grp .. 32*grp+31 of every block
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint8_t *row_base = panel + (t >> 3) * 1024 + (t & 7) * 128;
         const int swz = t & 7;
-        uint32_t sfull_uses = 0;                             // uses of s_full[half] by this thread
+        uint32_t sfull_uses[2] = {0, 0};                     // uses of s_full[0], s_full[1] by this thread
         bool ok = true;
 
         for (int tile = blockIdx.x, it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
@@ -356,16 +358,17 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 const uint32_t mk = (uint32_t)mult << k;
                 const uint32_t ck = (uint32_t)(uint64_t)((lo64 * mult + R) * ((int64_t)1 << k));
                 int ymax = 0;
-                for (int kb = half; ok && kb < kblocks; kb += 2) {
-                    ok = mbar_wait(smem_u32(&bars.s_full[half]), sfull_uses & 1, abortp, a.status);
+                for (int kb = 0; ok && kb < kblocks; ++kb) {
+                    const int sb = kb & 1;
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), sfull_uses[sb] & 1, abortp, a.status);
                     if (!ok) break;
-                    ++sfull_uses;
+                    ++sfull_uses[sb];
                     tcgen05_fence_after();
                     uint8_t *blk = row_base + kb * kPanelBlockBytes;
-#pragma unroll 1
-                    for (int j = 2 * side; j < 2 * side + 2; ++j) {
+                    {
+                        const int j = grp;
                         uint32_t acc[32];
-                        tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
+                        tmem_ld32(tmem + lane_addr + sb * 128 + j * 32, acc);
                         uint32_t w[8];
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
@@ -384,21 +387,22 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
                     }
                     tcgen05_fence_before();
-                    mbar_arrive(smem_u32(&bars.s_free[half]));
+                    mbar_arrive(smem_u32(&bars.s_free[sb]));
                 }
                 xmax = (int)((uint32_t)ymax * mk + ck) >> 24;
             } else {
                 const int32_t mult_hi = mult << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
-                for (int kb = half; ok && kb < kblocks; kb += 2) {
-                    ok = mbar_wait(smem_u32(&bars.s_full[half]), sfull_uses & 1, abortp, a.status);
+                for (int kb = 0; ok && kb < kblocks; ++kb) {
+                    const int sb = kb & 1;
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), sfull_uses[sb] & 1, abortp, a.status);
                     if (!ok) break;
-                    ++sfull_uses;
+                    ++sfull_uses[sb];
                     tcgen05_fence_after();
                     uint8_t *blk = row_base + kb * kPanelBlockBytes;
-#pragma unroll 1
-                    for (int j = 2 * side; j < 2 * side + 2; ++j) {
+                    {
+                        const int j = grp;
                         uint32_t acc[32];
-                        tmem_ld32(tmem + lane_addr + half * 128 + j * 32, acc);
+                        tmem_ld32(tmem + lane_addr + sb * 128 + j * 32, acc);
                         uint32_t w[8];
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
@@ -415,7 +419,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
                     }
                     tcgen05_fence_before();
-                    mbar_arrive(smem_u32(&bars.s_free[half]));
+                    mbar_arrive(smem_u32(&bars.s_free[sb]));
                 }
             }
             xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
@@ -427,13 +431,13 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int cm = th.D - xmax;
             const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
             uint32_t rsum = 0;
-            for (int kb = half; kb < kblocks; kb += 2) {
+            for (int kb = 0; kb < kblocks; ++kb) {
                 uint8_t *blk = row_base + kb * kPanelBlockBytes;
-                uint4 v[4];
+                uint4 v[2];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
+                for (int c = 0; c < 2; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((2 * grp + c) ^ swz) << 4));
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
                     uint32_t s2 = 0;
 #pragma unroll
@@ -444,7 +448,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
                     }
                     rsum += (s2 & 0xffffu) + (s2 >> 16);
-                    *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(blk + (((2 * grp + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
             part_sum[grp][t] = (int)rsum;
@@ -460,13 +464,13 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
 
             // ---- phase 3: probabilities from the stored closeness values, in place
-            for (int kb = half; kb < kblocks; kb += 2) {
+            for (int kb = 0; kb < kblocks; ++kb) {
                 uint8_t *blk = row_base + kb * kPanelBlockBytes;
-                uint4 v[4];
+                uint4 v[2];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((4 * side + c) ^ swz) << 4));
+                for (int c = 0; c < 2; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((2 * grp + c) ^ swz) << 4));
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
                     uint32_t o[4];
 #pragma unroll
@@ -484,12 +488,12 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                             q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
                         }
                         if (CAUSAL) {
-                            const int nb = nv - (kb * kTile + (4 * side + c) * 16 + 4 * k);
+                            const int nb = nv - (kb * kTile + (2 * grp + c) * 16 + 4 * k);
                             q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
                         }
                         o[k] = q;
                     }
-                    *reinterpret_cast<uint4 *>(blk + (((4 * side + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4 *>(blk + (((2 * grp + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
                 // the tensor core reads the panel through the async proxy: hand this block over
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
