@@ -103,8 +103,8 @@ hccs_status_t ensure_capacity(hccs_ctx *ctx, int32_t heads) {
     int32_t cap = heads < 64 ? 64 : heads;
     HCCS_CUDA(ctx, cudaMalloc(&ctx->d_table, sizeof(hccs::HeadEntry) * cap));
     HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_table, sizeof(hccs::HeadEntry) * cap, cudaHostAllocDefault));
-    HCCS_CUDA(ctx, cudaMalloc(&ctx->d_mult, sizeof(int32_t) * cap));
-    HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_mult, sizeof(int32_t) * cap, cudaHostAllocDefault));
+    HCCS_CUDA(ctx, cudaMalloc(&ctx->d_mult, sizeof(int32_t) * 4 * cap));
+    HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_mult, sizeof(int32_t) * 4 * cap, cudaHostAllocDefault));
     ctx->capacity = cap;
     return HCCS_OK;
 }
@@ -341,8 +341,30 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
     if (!g.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     HCCS_CUDA(ctx, cudaEventSynchronize(ctx->mult_copied));
-    memcpy(ctx->h_mult, requant_mult, sizeof(int32_t) * H);
-    HCCS_CUDA(ctx, cudaMemcpyAsync(ctx->d_mult, ctx->h_mult, sizeof(int32_t) * H,
+    // Per head: {multiplier, and for shifts up to 24 the constants of the single-multiply
+    // requantisation: multiplier << k, offset, -lo, hi - lo} (see hccs_fused.cu, phase 1).
+    for (int32_t h = 0; h < H; ++h) {
+        const int64_t M = requant_mult[h];
+        int32_t *e = ctx->h_mult + 4 * h;
+        e[0] = (int32_t)M;
+        e[1] = e[2] = e[3] = 0;
+        if (requant_shift <= 24) {
+            const int sh = requant_shift, k = 24 - sh;
+            const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
+            int64_t lo = -lim, hi = lim;
+            if (M > 0) {
+                lo = -((((int64_t)128 << sh) + R) / M);          // smallest accumulator that gives -128
+                hi = (((int64_t)128 << sh) - 1 - R) / M;         // largest accumulator that gives 127
+                if (lo < -lim) lo = -lim;
+                if (hi > lim) hi = lim;
+            }
+            e[0] = (int32_t)(uint32_t)((uint64_t)M << k);
+            e[1] = (int32_t)(uint32_t)(uint64_t)((lo * M + R) * ((int64_t)1 << k));
+            e[2] = (int32_t)-lo;
+            e[3] = (int32_t)(hi - lo);
+        }
+    }
+    HCCS_CUDA(ctx, cudaMemcpyAsync(ctx->d_mult, ctx->h_mult, sizeof(int32_t) * 4 * H,
                                    cudaMemcpyHostToDevice, stream));
     HCCS_CUDA(ctx, cudaEventRecord(ctx->mult_copied, stream));
     hccs::FusedArgs a;

@@ -325,7 +325,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int q0 = qt * kTile;
             const int kblocks = CAUSAL ? qt + 1 : nblk;
             const HeadEntry th = a.table[head];
-            const int32_t mult = a.requant_mult[head];
+            const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 4 * head);   // host-prepared constants
             const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
 
             // the previous tile's O rows were staged in the panel: their bulk copies must have
@@ -342,21 +342,12 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // clamp.  With y = clamp(acc - lo, 0, hi - lo) (one instruction) and k = 24 - sh,
             // t = y*(M << k) + ((lo*M + R) << k) lies in [-2^31, 2^31) and x is its top byte: one 32-bit
             // multiply-add per logit, no shift, and the bytes are picked up by the packing PRMTs.
-            // Shifts above 24 take the 64-bit multiply instead.
+            // The four constants come from the host, per head.  Shifts above 24 take the 64-bit
+            // multiply instead.
             int xmax = -128;
             if (a.requant_shift <= 24) {
-                const int sh = a.requant_shift, k = 24 - sh;
-                const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
-                int64_t lo64 = -lim, hi64 = lim;
-                if (mult > 0) {
-                    lo64 = -((((int64_t)128 << sh) + R) / mult);
-                    hi64 = (((int64_t)128 << sh) - 1 - R) / mult;
-                    lo64 = max(lo64, -lim);
-                    hi64 = min(hi64, lim);
-                }
-                const int neg_lo = (int)-lo64, span = (int)(hi64 - lo64);
-                const uint32_t mk = (uint32_t)mult << k;
-                const uint32_t ck = (uint32_t)(uint64_t)((lo64 * mult + R) * ((int64_t)1 << k));
+                const uint32_t mk = (uint32_t)rq.x, ck = (uint32_t)rq.y;
+                const int neg_lo = rq.z, span = rq.w;
                 int ymax = 0;
                 for (int kb = 0; ok && kb < kblocks; ++kb) {
                     const int sb = kb & 1;
@@ -391,7 +382,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 }
                 xmax = (int)((uint32_t)ymax * mk + ck) >> 24;
             } else {
-                const int32_t mult_hi = mult << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
+                const int32_t mult_hi = rq.x << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
                 for (int kb = 0; ok && kb < kblocks; ++kb) {
                     const int sb = kb & 1;
                     ok = mbar_wait(smem_u32(&bars.s_full[sb]), sfull_uses[sb] & 1, abortp, a.status);

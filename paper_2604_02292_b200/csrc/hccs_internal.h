@@ -46,7 +46,7 @@ struct FusedArgs {
     const int8_t *Q, *K, *V;
     int32_t *O;
     const HeadEntry *table;
-    const int32_t *requant_mult;   // device, H entries
+    const int32_t *requant_mult;   // device, 4 ints per head: see hccs_attention_fused in hccs_api.cu
     uint32_t *status;
     int32_t requant_shift;
     int32_t B, H, L, d;
