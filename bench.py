@@ -28,6 +28,11 @@ if ROOT not in sys.path:
 
 L2_BYTES = 126 * 1000 * 1000
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (cold L2, so part of the output had not been written back yet); None for workloads
+# that were not captured.  Set back to None when the kernel of a workload changes.
+NCU_TRAFFIC_BYTES = {"config2": 67.12e6 + 24.3e6, "config3": 33.57e6 + 0.7e6, "config4": 201.34e6 + 154.3e6,
+                     "config5": 75.6e6 + 52.7e6}
 NOMINAL_HBM_GBS = 8000.0
 METRIC = "hccs_forward rows/s (int8 logits -> uint8 probabilities, exact divide)"
 
@@ -229,7 +234,8 @@ def run_fused(args):
         "roofline": {"bound": "alu", "achieved": FUSED_ALU_OPS_PER_LOGIT * logits / (ms * 1e-3) / 1e12,
                      "peak": ALU_PEAK_TOPS, "unit": "Top/s",
                      "frac": FUSED_ALU_OPS_PER_LOGIT * logits / (ms * 1e-3) / 1e12 / ALU_PEAK_TOPS,
-                     "peak_kind": "derived: 148 SMs x 128 int lanes x 1.965 GHz", "traffic": None},
+                     "peak_kind": "derived: 148 SMs x 128 int lanes x 1.965 GHz",
+                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name)},
         "gpu_launches": int(launches), "clocks": clocks, "device_status": ctx.hccs_device_status(),
     }
     if full:
@@ -385,7 +391,7 @@ def run_ours(args):
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                         "traffic": None, "algorithmic_bytes_per_launch": flat,
+                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes_per_launch": flat,
                          "true_bytes_per_launch": true_bytes,
                          "achieved_true_bytes": true_bytes / kernel_s / 1e9},
             "e2e": {"value": e2e_rows_per_s, "unit": "rows/s", "h2d_bytes_per_step": nbytes,
