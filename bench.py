@@ -293,13 +293,17 @@ def run_ours(args):
     wl = workload_for(args)
     ctx = pkg.Context(local)
     ctx.hccs_params_upload(wl.theta, wl.n_design)
-    flags = wl.flags
+    extra = {"u8div": 0, "u8clb": pkg.HCCS_RECIP_CLB, "u16div": pkg.HCCS_OUT_U16,
+             "u16clb": pkg.HCCS_OUT_U16 | pkg.HCCS_RECIP_CLB}[args.mode]
+    flags = wl.flags | extra
+    osz = 2 if flags & pkg.HCCS_OUT_U16 else 1
+    odt = torch.uint16 if osz == 2 else torch.uint8
     nbytes = wl.elements
-    nbuf = max(4, -(-4 * L2_BYTES // (2 * nbytes)))
+    nbuf = max(4, -(-4 * L2_BYTES // ((1 + osz) * nbytes)))
     nbuf = min(nbuf, 64)
     host_x = torch.from_numpy(wl.logits).pin_memory()
     xs = [host_x.to(dev, non_blocking=True) for _ in range(nbuf)]
-    ps = [torch.empty(wl.logits.shape, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
+    ps = [torch.empty(wl.logits.shape, dtype=odt, device=dev) for _ in range(nbuf)]
     stream = torch.cuda.current_stream()
     sptr = stream.cuda_stream
     torch.cuda.synchronize()
@@ -344,7 +348,7 @@ def run_ours(args):
     rows_per_s = world * wl.rows / (ms_per_step * 1e-3)
 
     # ---------------- end to end: host tensors in, host tensors out, through hccs_forward_host
-    host_p = torch.empty(wl.logits.shape, dtype=torch.uint8).pin_memory()
+    host_p = torch.empty(wl.logits.shape, dtype=odt).pin_memory()
     e2e_steps = max(3, min(args.steps, 10)) if full else 0
     for _ in range(2 if full else 0):
         ctx.hccs_forward_host(host_x, host_p, xs[0], ps[0], flags, stream=sptr)
@@ -365,12 +369,13 @@ def run_ours(args):
     if rank == 0:
         peak, peak_kind = measured_peak()
         kernel_s = ms_per_step * 1e-3
-        flat = algorithmic_bytes(wl, True)
-        true_bytes = algorithmic_bytes(wl, False)
+        flat = algorithmic_bytes(wl, True) + (osz - 1) * wl.elements
+        true_bytes = algorithmic_bytes(wl, False) + (osz - 1) * wl.elements
         achieved = flat / kernel_s / 1e9
         # parity spot check of the timed launch configuration against the oracle (rank 0)
         from oracle import hccs_oracle as orc
-        mode = orc.MODE_CAUSAL if flags & 4 else 0
+        mode = (orc.MODE_CAUSAL if flags & 4 else 0) | (orc.MODE_U16 if flags & 1 else 0) | \
+            (orc.MODE_CLB if flags & 2 else 0)
         nb = max(1, wl.shape[0] // 64)
         want = orc.forward(wl.logits[:nb], wl.theta, mode, threads=os.cpu_count() or 1)
         mism = int((ps[0][:nb].cpu().numpy() != want).sum())
@@ -383,19 +388,20 @@ def run_ours(args):
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
             "data": "synthetic",
-            "config": {"workload": wl.name, "shape": list(wl.shape), "flags": flags,
+            "config": {"workload": wl.name, "shape": list(wl.shape), "flags": flags, "mode": args.mode,
                        "cache": f"rotating {nbuf} buffer sets ({2 * nbytes * nbuf >> 20} MiB) > L2",
                        "timing": "CUDA events around the K steps on the launching stream"},
             "elements_per_s": world * wl.elements / kernel_s,
-            "gbs_flat_2B_per_elem": achieved * world,
+            "gbs_algorithmic": achieved * world,
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes_per_launch": flat,
+                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name) if args.mode == "u8div" else None,
+                         "algorithmic_bytes_per_launch": flat,
                          "true_bytes_per_launch": true_bytes,
                          "achieved_true_bytes": true_bytes / kernel_s / 1e9},
             "e2e": {"value": e2e_rows_per_s, "unit": "rows/s", "h2d_bytes_per_step": nbytes,
-                    "d2h_bytes_per_step": nbytes,
+                    "d2h_bytes_per_step": nbytes * osz,
                     "ms_per_step": e2e_ms / e2e_steps if full else None, "steps": e2e_steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
@@ -420,6 +426,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--mode", default="u8div", choices=["u8div", "u8clb", "u16div", "u16clb"],
+                    help="output type and reciprocal of hccs_forward (the headline is u8div)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-resident timing (for profiler captures): no end-to-end leg, "
                          "no CPU baseline, no clock sampling")

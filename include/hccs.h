@@ -23,6 +23,8 @@
  *     the default stream) and the call returns without synchronising, unless
  *     stated otherwise.
  *   - Errors are return codes only.  On any error nothing is launched.
+ *   - A context is not thread-safe: one call at a time per context (different contexts, also on
+ *     the same device, are independent).
  *   - There is no CPU implementation behind this interface.
  */
 #ifndef HCCS_H

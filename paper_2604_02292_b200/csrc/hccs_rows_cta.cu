@@ -14,6 +14,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "hccs_device.cuh"
 #include "hccs_internal.h"
 
@@ -364,10 +366,12 @@ static __device__ __align__(256) uint32_t g_static_scratch[kStaticWords];
 
 constexpr int kStaticMaxDevices = 64;
 uint32_t *g_static_ptr[kStaticMaxDevices] = {};   // device address of the array, per device
+std::mutex g_static_mutex;
 
 // The array's name is only a host-side handle; the address the kernel can use has to be asked
 // for, once per device and with that device current.
 cudaError_t static_scratch_address(int device, uint32_t **out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_ptr[device]) {
         void *p = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);

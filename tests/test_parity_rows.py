@@ -76,11 +76,11 @@ def test_out_shift(ctx, oracle, hccs, out_shift):
             _check(ctx, oracle, wl, flags, out_shift=out_shift)
 
 
-@pytest.mark.parametrize("misalign", [1, 4, 8, 15])
+@pytest.mark.parametrize("misalign", [1, 4, 8, 15, 16, 48])
 def test_unaligned_pointers(ctx, oracle, hccs, misalign):
-    for Lk in (64, 128, 2048):
+    for Lk in (64, 128, 2048, 4096):
         wl = hccs.workloads.make_rows(9, (1, 2, 6, Lk), kind="gauss")
-        for flags in (0, 1):
+        for flags in (0, 1, 4):
             _check(ctx, oracle, wl, flags, misalign=misalign)
 
 
