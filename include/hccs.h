@@ -116,6 +116,19 @@ hccs_status_t hccs_forward(hccs_ctx_t *ctx, const int8_t *logits, void *probs,
                            uint32_t flags, void *cuda_stream);
 
 /*
+ * hccs_forward with a padding mask: key j of batch entry b takes part iff j < key_len[b] (and,
+ * with HCCS_CAUSAL, iff the causal rule holds as well).  This is the mask of the paper's encoder
+ * workloads, whose sequences are padded to 64 or 128 tokens (Section "Models and tasks"); the
+ * paper itself does not define masking: masked keys are left out of the max (Eq. 1) and the sum
+ * (Eq. 5) and produce 0, a row without valid keys produces zeros.
+ *   key_len  device int32 [B]; values are clamped to [0, Lk]
+ * Everything else as hccs_forward.
+ */
+hccs_status_t hccs_forward_keylen(hccs_ctx_t *ctx, const int8_t *logits, void *probs,
+                                  const int32_t *key_len, int32_t B, int32_t H, int32_t Lq, int32_t Lk,
+                                  uint32_t flags, void *cuda_stream);
+
+/*
  * The same operation for HOST tensors: copies `logits_host` to `logits_staging`, runs
  * hccs_forward, copies the result back to `probs_host`, all on `cuda_stream`, in pieces so that
  * the two copy directions and the kernel overlap.  The caller provides both device staging

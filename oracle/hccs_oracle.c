@@ -140,7 +140,8 @@ int64_t hccs_oracle_row(const int8_t *x, const uint8_t *valid, int64_t n,
 /*
  * Rows [row_begin, row_end) of a contiguous [Bt,H,Lq,Lk] int8 tensor.  The
  * head of flat row r is (r / Lq) mod H; params is H triples (B,S,D) as int32.
- * Causal: position j of query i is valid when j <= i + (Lk - Lq).
+ * Causal: position j of query i is valid when j <= i + (Lk - Lq).  key_len (optional): key j of
+ * batch entry b is valid when j < key_len[b] (padding mask; both rules combine).
  * probs is uint8 (u8 modes) or uint16 (u16 modes), same shape.
  * Returns 0, or -1 when a value would not fit the output type.
  */
@@ -148,7 +149,8 @@ int hccs_oracle_forward(const int8_t *logits, void *probs,
                         int64_t Bt, int64_t H, int64_t Lq, int64_t Lk,
                         const int32_t *params, int mode, int64_t out_shift,
                         int64_t row_begin, int64_t row_end,
-                        int64_t *p_tmp /* Lk */, uint8_t *valid_tmp /* Lk */)
+                        int64_t *p_tmp /* Lk */, uint8_t *valid_tmp /* Lk */,
+                        const int32_t *key_len /* Bt entries or NULL: padding mask */)
 {
     int64_t r, j;
     (void)Bt;
@@ -157,8 +159,14 @@ int hccs_oracle_forward(const int8_t *logits, void *probs,
         int64_t i = r % Lq;
         const int8_t *x = logits + r * Lk;
         const uint8_t *valid = NULL;
-        if (mode & ORACLE_MODE_CAUSAL) {
-            for (j = 0; j < Lk; ++j) valid_tmp[j] = (uint8_t)(j <= i + (Lk - Lq));
+        if ((mode & ORACLE_MODE_CAUSAL) || key_len) {
+            int64_t b = r / (Lq * H);
+            for (j = 0; j < Lk; ++j) {
+                int ok = 1;
+                if ((mode & ORACLE_MODE_CAUSAL) && !(j <= i + (Lk - Lq))) ok = 0;
+                if (key_len && !(j < (int64_t)key_len[b])) ok = 0;      /* key j is padding */
+                valid_tmp[j] = (uint8_t)ok;
+            }
             valid = valid_tmp;
         }
         hccs_oracle_row(x, valid, Lk, params[3 * h + 0], params[3 * h + 1], params[3 * h + 2],

@@ -58,7 +58,7 @@ def lib() -> ctypes.CDLL:
                                           _p, _p, _p]
             L.hccs_oracle_row.restype = _i64
             L.hccs_oracle_forward.argtypes = [_p, _p, _i64, _i64, _i64, _i64, _p, ctypes.c_int,
-                                              _i64, _i64, _i64, _p, _p]
+                                              _i64, _i64, _i64, _p, _p, _p]
             L.hccs_oracle_forward.restype = ctypes.c_int
             L.hccs_oracle_requant.argtypes = [_i64, _i64, _i64]
             L.hccs_oracle_requant.restype = _i64
@@ -109,11 +109,12 @@ def _params_array(params, H):
 
 
 def forward(logits, params, mode: int = 0, out_shift: int = 0, threads: int = 1,
-            row_range=None):
+            row_range=None, key_len=None):
     """HCCS over a contiguous int8 [B,H,Lq,Lk] array.  Returns uint8 / uint16, same shape.
 
     ``threads`` > 1 splits the independent rows over that many Python threads.
     ``row_range=(r0, r1)`` computes only those flat rows (the rest stay zero).
+    ``key_len`` (int32 [B]) is the padding mask: key j of batch entry b is valid iff j < key_len[b].
     """
     x = np.ascontiguousarray(logits, dtype=np.int8)
     Bt, H, Lq, Lk = x.shape
@@ -121,12 +122,15 @@ def forward(logits, params, mode: int = 0, out_shift: int = 0, threads: int = 1,
     out = np.zeros(x.shape, dtype=np.uint16 if (mode & MODE_U16) else np.uint8)
     r0, r1 = (0, Bt * H * Lq) if row_range is None else row_range
     L = lib()
+    kl = None if key_len is None else np.ascontiguousarray(key_len, dtype=np.int32)
+    if kl is not None and kl.shape != (Bt,):
+        raise ValueError("key_len must have one entry per batch entry")
 
     def work(a, b):
         p_tmp = np.zeros(max(Lk, 1), dtype=np.int64)
         v_tmp = np.zeros(max(Lk, 1), dtype=np.uint8)
         rc = L.hccs_oracle_forward(_ptr(x), _ptr(out), Bt, H, Lq, Lk, _ptr(pa), mode,
-                                   out_shift, a, b, _ptr(p_tmp), _ptr(v_tmp))
+                                   out_shift, a, b, _ptr(p_tmp), _ptr(v_tmp), _ptr(kl))
         if rc != 0:
             raise OverflowError("oracle output does not fit the output type")
 

@@ -35,7 +35,8 @@ HCCS_RECIP_DIV = 0
 HCCS_RECIP_CLB = 2
 HCCS_CAUSAL = 4
 
-EXPORTS = ("hccs_create", "hccs_destroy", "hccs_params_check", "hccs_params_upload", "hccs_forward", "hccs_forward_host",
+EXPORTS = ("hccs_create", "hccs_destroy", "hccs_params_check", "hccs_params_upload", "hccs_forward",
+           "hccs_forward_keylen", "hccs_forward_host",
            "hccs_attention_fused", "hccs_device_status", "hccs_last_cuda_error", "hccs_status_string",
            "hccs_launch_count", "hccs_forward_static_scratch")
 
@@ -51,6 +52,8 @@ _lib.hccs_params_check.argtypes = [_vp, _i32, _i32, ctypes.POINTER(_i32)]
 _lib.hccs_params_check.restype = ctypes.c_int
 _lib.hccs_forward.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _u32, _vp]
 _lib.hccs_forward.restype = ctypes.c_int
+_lib.hccs_forward_keylen.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _u32, _vp]
+_lib.hccs_forward_keylen.restype = ctypes.c_int
 _lib.hccs_forward_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _u32, _vp]
 _lib.hccs_forward_host.restype = ctypes.c_int
 _lib.hccs_attention_fused.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
@@ -142,6 +145,17 @@ class Context:
                                _stream_ptr(stream))
         if st != HCCS_OK:
             raise HccsError(st, "hccs_forward")
+
+    # -- hccs_forward_keylen
+    def hccs_forward_keylen(self, logits, probs, key_len, flags: int = 0, stream=None) -> None:
+        B, H, Lq, Lk = logits.shape
+        _check_tensor(logits, "logits", 1)
+        _check_tensor(probs, "probs", 2 if flags & HCCS_OUT_U16 else 1, logits.shape)
+        _check_tensor(key_len, "key_len", 4, (B,))
+        st = _lib.hccs_forward_keylen(self._h, _ptr(logits), _ptr(probs), _ptr(key_len), B, H, Lq, Lk,
+                                      int(flags), _stream_ptr(stream))
+        if st != HCCS_OK:
+            raise HccsError(st, "hccs_forward_keylen")
 
     # -- hccs_forward_host
     def hccs_forward_host(self, logits_host, probs_host, logits_staging, probs_staging,

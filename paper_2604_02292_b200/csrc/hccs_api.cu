@@ -123,7 +123,8 @@ hccs_status_t check_forward_args(hccs_ctx *ctx, const void *in, const void *out,
     return HCCS_OK;
 }
 
-hccs::RowArgs make_row_args(const hccs_ctx *ctx, int32_t rows, int32_t H, int32_t Lq, int32_t Lk) {
+hccs::RowArgs make_row_args(const hccs_ctx *ctx, int32_t rows, int32_t H, int32_t Lq, int32_t Lk, uint32_t flags,
+                            const int32_t *key_len) {
     hccs::RowArgs a;
     a.table = ctx->d_table;
     a.status = ctx->d_status;
@@ -133,6 +134,8 @@ hccs::RowArgs make_row_args(const hccs_ctx *ctx, int32_t rows, int32_t H, int32_
     a.Lq = Lq;
     a.Lk = Lk;
     a.causal_off = Lk - Lq;
+    a.causal = (flags & HCCS_CAUSAL) ? 1 : 0;
+    a.key_len = key_len;
     a.out_shift = ctx->out_shift;
     a.slice0 = 0;
     a.div_Lq = hccs::make_fastdiv((uint32_t)Lq);
@@ -257,7 +260,23 @@ hccs_status_t hccs_forward(hccs_ctx_t *ctx, const int8_t *logits, void *probs,
     if ((flags & HCCS_OUT_U16) && (const void *)logits == probs) return HCCS_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);
     if (!g.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
-    hccs::RowArgs a = make_row_args(ctx, (int32_t)rows, H, Lq, Lk);
+    hccs::RowArgs a = make_row_args(ctx, (int32_t)rows, H, Lq, Lk, flags, nullptr);
+    HCCS_CUDA(ctx, hccs::launch_rows(logits, probs, a, flags, (cudaStream_t)cuda_stream, &ctx->launches));
+    return HCCS_OK;
+}
+
+hccs_status_t hccs_forward_keylen(hccs_ctx_t *ctx, const int8_t *logits, void *probs, const int32_t *key_len,
+                                  int32_t B, int32_t H, int32_t Lq, int32_t Lk,
+                                  uint32_t flags, void *cuda_stream) {
+    hccs_status_t st = check_forward_args(ctx, logits, probs, B, H, Lq, Lk, flags);
+    if (st != HCCS_OK) return st;
+    const int64_t rows = (int64_t)B * H * Lq;
+    if (rows * Lk == 0) return HCCS_OK;
+    if (!key_len) return HCCS_ERR_INVALID_ARG;
+    if ((flags & HCCS_OUT_U16) && (const void *)logits == probs) return HCCS_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+    hccs::RowArgs a = make_row_args(ctx, (int32_t)rows, H, Lq, Lk, flags, key_len);
     HCCS_CUDA(ctx, hccs::launch_rows(logits, probs, a, flags, (cudaStream_t)cuda_stream, &ctx->launches));
     return HCCS_OK;
 }
@@ -301,8 +320,8 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
         // a piece starts at slice s0: rotate the head index by running the kernel on a view whose
         // flat row 0 is that slice; (r / Lq) mod H then needs the slice offset folded in, which
         // the row arguments carry as a starting slice
-        hccs::RowArgs a = make_row_args(ctx, (int32_t)((s1 - s0) * Lq), H, Lq, Lk);
-        a.slice0 = (int32_t)(s0 % H);
+        hccs::RowArgs a = make_row_args(ctx, (int32_t)((s1 - s0) * Lq), H, Lq, Lk, flags, nullptr);
+        a.slice0 = (int32_t)s0;
         HCCS_CUDA(ctx, hccs::launch_rows(logits_staging + off, (char *)probs_staging + off * osz, a,
                                          flags, stream, &ctx->launches));
         HCCS_CUDA(ctx, cudaEventRecord(ctx->ev_done[p], stream));

@@ -14,12 +14,13 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv &f) {
     return (__umulhi(n, f.mul) + n) >> f.shift;
 }
 
-// (head, query index) of flat row r: head = ((r / Lq) + slice0) mod H, i = r mod Lq.
-__device__ __forceinline__ void row_coords(uint32_t r, const RowArgs &a, uint32_t &head, uint32_t &i) {
+// (batch entry, head, query index) of flat row r: slice = r / Lq + slice0, b = slice / H,
+// head = slice mod H, i = r mod Lq.
+__device__ __forceinline__ void row_coords(uint32_t r, const RowArgs &a, uint32_t &b, uint32_t &head, uint32_t &i) {
     uint32_t bh = fast_div(r, a.div_Lq);
     i = r - bh * (uint32_t)a.Lq;
     bh += (uint32_t)a.slice0;
-    uint32_t b = fast_div(bh, a.div_H);
+    b = fast_div(bh, a.div_H);
     head = bh - b * (uint32_t)a.H;
 }
 
@@ -45,12 +46,18 @@ __device__ __forceinline__ uint32_t reciprocal(uint32_t Z) {
     return q + (rem >= Z ? 1u : 0u);
 }
 
-// Number of valid keys of query i (a prefix of the row).
-template <bool CAUSAL>
-__device__ __forceinline__ int valid_keys(uint32_t i, const RowArgs &a) {
-    if (!CAUSAL) return a.Lk;
-    int nv = (int)i + a.causal_off + 1;
-    return min(max(nv, 0), a.Lk);
+// Number of valid keys of query i of batch entry b: always a prefix of the row.  MASKED kernels
+// apply the causal rule (when a.causal) and the per-batch key length (when a.key_len is set).
+template <bool MASKED>
+__device__ __forceinline__ int valid_keys_causal(uint32_t i, const RowArgs &a) {
+    if (!MASKED || !a.causal) return a.Lk;
+    return min(max((int)i + a.causal_off + 1, 0), a.Lk);
+}
+template <bool MASKED>
+__device__ __forceinline__ int valid_keys(uint32_t b, uint32_t i, const RowArgs &a) {
+    int nv = valid_keys_causal<MASKED>(i, a);
+    if (MASKED && a.key_len) nv = min(nv, max(a.key_len[b], 0));   // reads global memory
+    return nv;
 }
 
 }  // namespace hccs

@@ -31,8 +31,10 @@ struct RowArgs {
     int32_t rows;             // B*H*Lq
     int32_t H, Lq, Lk;
     int32_t causal_off;       // Lk - Lq
+    int32_t causal;           // 1: key j of query i valid iff j <= i + causal_off
+    const int32_t *key_len;   // device, one entry per batch entry, or NULL: keys beyond key_len[b] are padding
     int32_t out_shift;        // OUT_SHIFT of Eq. 8
-    int32_t slice0;           // (b*H + h) index of flat row 0, mod H (views that start mid-tensor)
+    int32_t slice0;           // b*H + h of flat row 0 (views that start mid-tensor)
     FastDiv div_Lq, div_H;
 };
 

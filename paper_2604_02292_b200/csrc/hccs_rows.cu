@@ -40,10 +40,10 @@ __global__ void __launch_bounds__(256) rows_generic_kernel(const int8_t *__restr
     const int warps_per_block = blockDim.x >> 5;
     for (int64_t r = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); r < a.rows;
          r += (int64_t)gridDim.x * warps_per_block) {
-        uint32_t head, i;
-        row_coords((uint32_t)r, a, head, i);
+        uint32_t b, head, i;
+        row_coords((uint32_t)r, a, b, head, i);
         const HeadEntry th = a.table[head];
-        const int nv = valid_keys<CAUSAL>(i, a);
+        const int nv = valid_keys<CAUSAL>(b, i, a);
         const int8_t *x = x_all + r * a.Lk;
         // pass 1: m = max over the valid keys (Eq. 1)
         int m = -128;
@@ -108,9 +108,9 @@ __global__ void __launch_bounds__(256) rows_lanegroup_kernel(const int8_t *__res
         const uint32_t r = (uint32_t)(slab0 + u) * ROWS_PER_SLAB + lane / G;
         rowid[u] = r;
         const bool live = (slab0 + u) < slabs && r < (uint32_t)a.rows;
-        uint32_t head = 0, i = 0;
-        if (live) row_coords(r, a, head, i);
-        nv[u] = live ? valid_keys<CAUSAL>(i, a) : 0;
+        uint32_t b = 0, head = 0, i = 0;
+        if (live) row_coords(r, a, b, head, i);
+        nv[u] = live ? valid_keys<CAUSAL>(b, i, a) : 0;
         th[u] = a.table[head];
 #pragma unroll
         for (int v = 0; v < V; ++v) {
@@ -289,7 +289,8 @@ cudaError_t launch_mode(const int8_t *x, void *p, const RowArgs &a, cudaStream_t
 cudaError_t launch_rows(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                         cudaStream_t stream, uint64_t *launches) {
     cudaError_t e;
-    switch (flags & 7u) {
+    const uint32_t sel = (flags & 3u) | (((flags & 4u) || a.key_len) ? 4u : 0u);   // bit 2: any masking
+    switch (sel) {
         case 0: e = launch_mode<false, false, false>(logits, probs, a, stream); break;
         case 1: e = launch_mode<true, false, false>(logits, probs, a, stream); break;
         case 2: e = launch_mode<false, true, false>(logits, probs, a, stream); break;

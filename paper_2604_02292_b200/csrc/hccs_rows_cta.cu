@@ -127,9 +127,9 @@ __global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all,
         if (j.row >= a.rows) {
             j.row = -1;
         } else {
-            uint32_t qi;
-            row_coords((uint32_t)j.row, a, j.head, qi);
-            j.nv = valid_keys<CAUSAL>(qi, a);
+            uint32_t b, qi;
+            row_coords((uint32_t)j.row, a, b, j.head, qi);
+            j.nv = valid_keys<CAUSAL>(b, qi, a);
             j.bytes = (uint32_t)((j.nv + 15) & ~15);
             if (j.bytes) {
                 mbar_expect_tx(bar[s], j.bytes);
@@ -440,6 +440,8 @@ extern "C" hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *p
     a.Lq = Lq;
     a.Lk = Lk;
     a.causal_off = Lk - Lq;
+    a.causal = (flags & HCCS_CAUSAL) ? 1 : 0;
+    a.key_len = nullptr;
     a.out_shift = out_shift;
     a.slice0 = 0;
     a.div_Lq = hccs::make_fastdiv((uint32_t)Lq);

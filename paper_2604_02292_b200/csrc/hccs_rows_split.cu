@@ -77,14 +77,15 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     const int sub = lane % G;
     const uint32_t row = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RW + lane / G;
     const bool live = row < (uint32_t)a.rows;
-    uint32_t head = 0, qi = 0;
-    if (live) row_coords(row, a, head, qi);
-    const int nv = live ? valid_keys<CAUSAL>(qi, a) : 0;
+    uint32_t bidx = 0, head = 0, qi = 0;
+    if (live) row_coords(row, a, bidx, head, qi);
+    int nv = live ? valid_keys_causal<CAUSAL>(qi, a) : 0;
     // Programmatic dependent launch: everything above touches no global memory, so it may run
     // while the previous kernel in the stream drains; all reads and writes come after the wait.
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const HeadEntry th = a.table[head];
+    if (CAUSAL && a.key_len && live) nv = min(nv, max(a.key_len[bidx], 0));   // padding mask
 
     // Causal: a chunk index v whose columns lie beyond every row of this warp is skipped
     // altogether (warp-uniform), e.g. the right half of the first 64 queries of a 128-key head.

@@ -300,6 +300,25 @@ def test_forward_head_indexing_and_causal_alignment():
     assert (part[7:19] == a.reshape(-1, Lk)[7:19]).all() and not part[:7].any() and not part[19:].any()
 
 
+def test_forward_key_length_mask():
+    """Padding mask: key j of batch entry b is valid iff j < key_len[b]; combined with causal."""
+    rng = np.random.default_rng(8)
+    Bt, H, Lq, Lk = 4, 3, 5, 7
+    theta = np.array([(4000 - 500 * h, h + 1, 9 + 2 * h) for h in range(H)], dtype=np.int32)
+    x = rng.integers(-128, 128, size=(Bt, H, Lq, Lk)).astype(np.int8)
+    key_len = np.array([7, 3, 0, 1], dtype=np.int32)
+    for mode in (0, orc.MODE_U16 | orc.MODE_CLB, orc.MODE_CAUSAL):
+        out = orc.forward(x, theta, mode, key_len=key_len)
+        for b, h, i in np.ndindex(Bt, H, Lq):
+            valid = [1 if j < key_len[b] and (not mode & orc.MODE_CAUSAL or j <= i + (Lk - Lq)) else 0
+                     for j in range(Lk)]
+            want = big.hccs_row(x[b, h, i].tolist(), theta[h], u16=bool(mode & 1), clb=bool(mode & 2), valid=valid)
+            assert out[b, h, i].tolist() == want
+    assert not out[2].any()                                     # a batch entry of length 0 gives zeros
+    full = orc.forward(x, theta, 0, key_len=np.full(Bt, Lk, np.int32))
+    assert (full == orc.forward(x, theta, 0)).all()             # full lengths = no mask
+
+
 # ----------------------------------------------------------------- constraints
 def test_constraints_one_at_a_time():
     n = 64

@@ -138,6 +138,29 @@ def test_every_row_sum_is_reached(ctx, oracle, hccs):
     assert set(range(383, 32705)) <= reached
 
 
+@pytest.mark.parametrize("Lk", [16, 33, 64, 128, 176, 512, 1024, 2048, 4096])
+def test_key_length_mask(ctx, oracle, hccs, Lk):
+    """hccs_forward_keylen: the padding mask of encoder workloads, alone and with the causal rule."""
+    import torch
+    Bt, H, Lq = 9, 3, 6
+    wl = hccs.workloads.make_rows(300 + Lk, (Bt, H, Lq, Lk), kind="gauss")
+    rng = np.random.default_rng(Lk)
+    key_len = rng.integers(1, Lk + 1, size=Bt).astype(np.int32)
+    key_len[:4] = (0, Lk, Lk + 5, -3)                            # empty, full, beyond the row, negative
+    ctx.hccs_params_upload(wl.theta, wl.n_design)
+    x = torch.from_numpy(wl.logits).cuda()
+    kl = torch.from_numpy(key_len).cuda()
+    for flags in (0, 1, 2, 4, 5):
+        odt = torch.uint16 if flags & 1 else torch.uint8
+        p = torch.full(wl.logits.shape, 0x5A, dtype=odt, device="cuda")
+        ctx.hccs_forward_keylen(x, p, kl, flags)
+        torch.cuda.synchronize()
+        want = oracle.forward(wl.logits, wl.theta, oracle_mode(oracle, flags), threads=4,
+                              key_len=np.clip(key_len, 0, Lk))
+        assert_same(p.cpu().numpy(), want, f"keylen Lk={Lk} flags={flags}")
+    assert ctx.hccs_device_status() == 0
+
+
 def test_empty_tensors_and_errors(ctx, hccs):
     import torch
     ctx.hccs_params_upload([(300, 3, 85)] * 4, 64)
