@@ -103,6 +103,11 @@ class ClockSampler:
 
 def workload_for(args):
     from paper_2604_02292_b200 import workloads
+    if args.shape:
+        shape = tuple(int(v) for v in args.shape.split(","))
+        wl = workloads.make_rows(12345, shape, kind="gauss")
+        wl.name = "rows" + "x".join(str(v) for v in shape)
+        return wl
     return workloads.make_config(args.config)
 
 
@@ -426,6 +431,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--shape", default="", help="B,H,Lq,Lk: time hccs_forward on seeded Gaussian rows of this "
+                                                "shape instead of a named workload")
     ap.add_argument("--mode", default="u8div", choices=["u8div", "u8clb", "u16div", "u16clb"],
                     help="output type and reciprocal of hccs_forward (the headline is u8div)")
     ap.add_argument("--kernel-only", action="store_true",

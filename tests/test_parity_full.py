@@ -25,3 +25,27 @@ def test_full_size_config(hccs, oracle, c):
         del p
     assert ctx.hccs_device_status() == 0
     ctx.close()
+
+
+def test_tensor_beyond_4_gib(hccs, oracle):
+    """Byte offsets above 2^32: a [B,1,Lq,2048] tensor of 4.5 GiB built by repeating a seeded block;
+    rows on both sides of the 4 GiB line must equal the oracle's rows of the block."""
+    import torch
+    Lk, H, Lq = 2048, 1, 512
+    wl = hccs.workloads.make_rows(77, (64, H, Lq, Lk), kind="gauss")        # 64 MiB block
+    reps = 72                                                               # 4.5 GiB
+    ctx = hccs.Context(0)
+    ctx.hccs_params_upload(wl.theta, wl.n_design)
+    block = torch.from_numpy(wl.logits).cuda()
+    x = block.repeat(reps, 1, 1, 1)
+    assert x.numel() > 2 ** 32
+    p = torch.empty(x.shape, dtype=torch.uint8, device="cuda")
+    ctx.hccs_forward(x, p, 0)
+    torch.cuda.synchronize()
+    want = torch.from_numpy(oracle.forward(wl.logits, wl.theta, 0, threads=8)).cuda()
+    for rep in (0, 31, 63, 64, 65, reps - 1):                               # 64 * 64 MiB = 4 GiB
+        assert torch.equal(p[rep * 64:(rep + 1) * 64], want), f"repetition {rep}"
+    del x, p
+    # the same through the causal kernel on the tail block only would need Lq == Lk; use key lengths
+    assert ctx.hccs_device_status() == 0
+    ctx.close()
