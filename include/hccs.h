@@ -161,6 +161,18 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
                                    int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
                                    uint32_t flags, void *cuda_stream);
 
+/*
+ * hccs_attention_fused with a dequantised fp32 output: O[b,h,i,:] = float(int32 accumulator) *
+ * out_scale[h] (HOST float [H]; e.g. the V quantisation step divided by 255).  The integer result
+ * is exact; the two fp32 roundings keep the relative error below 2^-23.  O is device float
+ * [B, H, L, d]; everything else as hccs_attention_fused.  (Not in the paper.)
+ */
+hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                       const int8_t *V, float *O, const float *out_scale,
+                                       const int32_t *requant_mult, int32_t requant_shift,
+                                       int32_t B, int32_t H, int32_t L, int32_t d,
+                                       uint32_t flags, void *cuda_stream);
+
 /* Reads (and clears) the device status word: 0 = no kernel gave up a bounded wait.  Synchronises
  * `cuda_stream`.  Returns HCCS_ERR_DEVICE_TIMEOUT when the word was non-zero; *word (may be NULL)
  * receives it. */

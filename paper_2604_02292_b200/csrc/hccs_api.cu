@@ -103,8 +103,8 @@ hccs_status_t ensure_capacity(hccs_ctx *ctx, int32_t heads) {
     int32_t cap = heads < 64 ? 64 : heads;
     HCCS_CUDA(ctx, cudaMalloc(&ctx->d_table, sizeof(hccs::HeadEntry) * cap));
     HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_table, sizeof(hccs::HeadEntry) * cap, cudaHostAllocDefault));
-    HCCS_CUDA(ctx, cudaMalloc(&ctx->d_mult, sizeof(int32_t) * 4 * cap));
-    HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_mult, sizeof(int32_t) * 4 * cap, cudaHostAllocDefault));
+    HCCS_CUDA(ctx, cudaMalloc(&ctx->d_mult, sizeof(int32_t) * 8 * cap));
+    HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_mult, sizeof(int32_t) * 8 * cap, cudaHostAllocDefault));
     ctx->capacity = cap;
     return HCCS_OK;
 }
@@ -335,10 +335,11 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
     return HCCS_OK;
 }
 
-hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
-                                   const int8_t *V, int32_t *O, const int32_t *requant_mult,
-                                   int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
-                                   uint32_t flags, void *cuda_stream) {
+// Shared by the int32 and the fp32 entry points: out_scale == NULL means int32 output.
+static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K, const int8_t *V, void *O,
+                                  const float *out_scale, const int32_t *requant_mult,
+                                  int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
+                                  uint32_t flags, void *cuda_stream) {
     if (!ctx || B < 0 || H < 0 || L < 0 || d < 0) return HCCS_ERR_INVALID_ARG;
     if (flags & ~7u) return HCCS_ERR_INVALID_ARG;
     if (flags & HCCS_OUT_U16) return HCCS_ERR_UNSUPPORTED;
@@ -361,12 +362,15 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     HCCS_CUDA(ctx, cudaEventSynchronize(ctx->mult_copied));
     // Per head: {multiplier, and for shifts up to 24 the constants of the single-multiply
-    // requantisation: multiplier << k, offset, -lo, hi - lo} (see hccs_fused.cu, phase 1).
+    // requantisation: multiplier << k, offset, -lo, hi - lo} (see hccs_fused.cu, phase 1), then the
+    // fp32 output scale; eight 32-bit words per head.
     for (int32_t h = 0; h < H; ++h) {
         const int64_t M = requant_mult[h];
-        int32_t *e = ctx->h_mult + 4 * h;
+        int32_t *e = ctx->h_mult + 8 * h;
         e[0] = (int32_t)M;
-        e[1] = e[2] = e[3] = 0;
+        e[1] = e[2] = e[3] = e[5] = e[6] = e[7] = 0;
+        const float scale = out_scale ? out_scale[h] : 1.0f;
+        memcpy(&e[4], &scale, sizeof(float));
         if (requant_shift <= 24) {
             const int sh = requant_shift, k = 24 - sh;
             const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
@@ -383,7 +387,7 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
             e[3] = (int32_t)(hi - lo);
         }
     }
-    HCCS_CUDA(ctx, cudaMemcpyAsync(ctx->d_mult, ctx->h_mult, sizeof(int32_t) * 4 * H,
+    HCCS_CUDA(ctx, cudaMemcpyAsync(ctx->d_mult, ctx->h_mult, sizeof(int32_t) * 8 * H,
                                    cudaMemcpyHostToDevice, stream));
     HCCS_CUDA(ctx, cudaEventRecord(ctx->mult_copied, stream));
     hccs::FusedArgs a;
@@ -391,12 +395,29 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
     a.table = ctx->d_table;
     a.requant_mult = ctx->d_mult;
     a.status = ctx->d_status;
-        a.requant_shift = requant_shift;
+    a.out_f32 = out_scale ? 1 : 0;
+    a.requant_shift = requant_shift;
     a.B = B; a.H = H; a.L = L; a.d = d;
     a.out_shift = ctx->out_shift;
     a.flags = flags;
     HCCS_CUDA(ctx, hccs::launch_fused(a, stream, &ctx->launches));
     return HCCS_OK;
+}
+
+hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                   const int8_t *V, int32_t *O, const int32_t *requant_mult,
+                                   int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
+                                   uint32_t flags, void *cuda_stream) {
+    return fused_common(ctx, Q, K, V, O, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+}
+
+hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                       const int8_t *V, float *O, const float *out_scale,
+                                       const int32_t *requant_mult, int32_t requant_shift,
+                                       int32_t B, int32_t H, int32_t L, int32_t d,
+                                       uint32_t flags, void *cuda_stream) {
+    if (!out_scale) return HCCS_ERR_INVALID_ARG;
+    return fused_common(ctx, Q, K, V, O, out_scale, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
 }
 
 hccs_status_t hccs_device_status(hccs_ctx_t *ctx, uint32_t *word, void *cuda_stream) {

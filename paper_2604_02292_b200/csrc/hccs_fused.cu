@@ -325,7 +325,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int q0 = qt * kTile;
             const int kblocks = CAUSAL ? qt + 1 : nblk;
             const HeadEntry th = a.table[head];
-            const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 4 * head);   // host-prepared constants
+            const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head);   // host-prepared constants
+            const float out_scale = __int_as_float(a.requant_mult[8 * head + 4]);
             const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
 
             // the previous tile's O rows were staged in the panel: their bulk copies must have
@@ -501,6 +502,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 tcgen05_fence_after();
                 uint32_t acc[16];
                 tmem_ld16(tmem + lane_addr + 256 + grp * 16, acc);
+                if (a.out_f32) {                                  // optional dequantised view of O
+#pragma unroll
+                    for (int g = 0; g < 16; ++g) acc[g] = __float_as_uint(__int2float_rn((int)acc[g]) * out_scale);
+                }
                 uint8_t *o_stage = panel + t * 272;
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
@@ -512,7 +517,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if (tid == 0) leave_flag = *abortp;                   // one reader, so that all row threads agree
             asm volatile("bar.sync 1, 512;" ::: "memory");
             if (ok && grp == 0) {
-                int32_t *o_row = a.O + ((int64_t)bh * a.L + q0 + t) * kD;
+                int32_t *o_row = (int32_t *)a.O + ((int64_t)bh * a.L + q0 + t) * kD;
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(o_row),
                              "r"(s_p + t * 272)
                              : "memory");

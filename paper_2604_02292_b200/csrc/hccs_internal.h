@@ -46,9 +46,10 @@ enum : uint32_t {
 
 struct FusedArgs {
     const int8_t *Q, *K, *V;
-    int32_t *O;
+    void *O;                       // int32 [B,H,L,d], or float when out_f32
     const HeadEntry *table;
-    const int32_t *requant_mult;   // device, 4 ints per head: see hccs_attention_fused in hccs_api.cu
+    const int32_t *requant_mult;   // device, 8 words per head: see fused_common in hccs_api.cu
+    int32_t out_f32;               // 1: O = float(acc) * scale_h
     uint32_t *status;
     int32_t requant_shift;
     int32_t B, H, L, d;

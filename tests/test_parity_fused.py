@@ -86,3 +86,28 @@ def test_unsupported_shapes_are_refused(hccs):
         ctx.hccs_attention_fused(q, q, q, o, [1000, 1000], 20, hccs.HCCS_OUT_U16)
     assert ei.value.status == hccs.HCCS_ERR_UNSUPPORTED
     ctx.close()
+
+
+def test_fp32_dequantised_output(hccs, oracle):
+    """O_f32 = float(int32 O) * scale_h: within 1e-6 relative of the exact product (fp64 from the oracle)."""
+    import torch
+    rng = np.random.default_rng(9)
+    Bt, H, L, d = 1, 3, 384, 64
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
+    theta = hccs.workloads.sample_theta(rng, H, L)
+    mult = rng.integers(768, 3841, size=H).astype(np.int32)
+    scale = np.array([0.03125 / 255, 1.7e-3, 0.4], dtype=np.float32)
+    ctx = hccs.Context(0)
+    ctx.hccs_params_upload(theta, L)
+    dQ, dK, dV = (torch.from_numpy(a).cuda() for a in (Q, K, V))
+    O = torch.empty(Q.shape, dtype=torch.float32, device="cuda")
+    ctx.hccs_attention_fused_f32(dQ, dK, dV, O, scale, mult, 20, 0)
+    torch.cuda.synchronize()
+    assert ctx.hccs_device_status() == 0
+    want = oracle.attention(Q, K, V, mult, 20, theta, 0, threads=8).astype(np.float64) * \
+        scale.astype(np.float64).reshape(1, H, 1, 1)
+    got = O.cpu().numpy().astype(np.float64)
+    err = np.abs(got - want)
+    assert (err <= 1e-6 * np.abs(want)).all(), float((err / np.maximum(np.abs(want), 1e-300)).max())
+    assert np.abs(want).max() > 0
+    ctx.close()
