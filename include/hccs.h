@@ -173,6 +173,30 @@ hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const i
                                        int32_t B, int32_t H, int32_t L, int32_t d,
                                        uint32_t flags, void *cuda_stream);
 
+/* A bounded grid of candidates for hccs_calibrate: D = D_lo, D_lo + D_step, ... <= D_hi (clipped to
+ * 1..127), S likewise (clipped to 0..127), and for each (D, S) the values B = S*D + ceil(256/n),
+ * + B_step, ... <= floor(32767/n): every candidate lies in the admissible band (Eq. 11). */
+typedef struct {
+    int32_t D_lo, D_hi, D_step;
+    int32_t S_lo, S_hi, S_step;
+    int32_t B_step;
+} hccs_calib_grid_t;
+
+/*
+ * Offline per-head calibration (Section "Offline Calibration", Eq. 10): scans the grid and returns,
+ * for each head, the theta that minimises the mean over the head's rows of
+ * KL( softmax(alpha * x) || q ), q the int16-path HCCS row renormalised to sum one (the paper
+ * recommends the int16 space; the renormalisation and the logit scale alpha are readings).
+ *   logits   device int8 [B, H, Lq, Lk], the calibration rows; n_design = Lk
+ *   best     HOST array of H triples (output);  best_kl  HOST double [H] (output, may be NULL)
+ * Ties go to the smallest (Dmax, S, B).  Needs no context.  Offline tooling: allocates and frees
+ * its work space (128 * B * H * Lq * 4 bytes plus small tables) and synchronises `cuda_stream`.
+ * fp64 throughout.  HCCS_ERR_CONSTRAINT when the grid holds no admissible candidate.
+ */
+hccs_status_t hccs_calibrate(const int8_t *logits, int32_t B, int32_t H, int32_t Lq, int32_t Lk,
+                             double alpha, const hccs_calib_grid_t *grid, hccs_head_params_t *best,
+                             double *best_kl, void *cuda_stream);
+
 /* Reads (and clears) the device status word: 0 = no kernel gave up a bounded wait.  Synchronises
  * `cuda_stream`.  Returns HCCS_ERR_DEVICE_TIMEOUT when the word was non-zero; *word (may be NULL)
  * receives it. */

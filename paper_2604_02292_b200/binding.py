@@ -38,7 +38,7 @@ HCCS_CAUSAL = 4
 EXPORTS = ("hccs_create", "hccs_destroy", "hccs_params_check", "hccs_params_upload", "hccs_forward",
            "hccs_forward_keylen", "hccs_forward_host",
            "hccs_attention_fused", "hccs_attention_fused_f32", "hccs_device_status", "hccs_last_cuda_error", "hccs_status_string",
-           "hccs_launch_count", "hccs_forward_static_scratch")
+           "hccs_launch_count", "hccs_forward_static_scratch", "hccs_calibrate")
 
 _vp, _i32, _u32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32
 
@@ -75,6 +75,29 @@ _lib.hccs_launch_count.restype = ctypes.c_uint64
 _lib.hccs_forward_static_scratch.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _i32, _u32,
                                              ctypes.POINTER(_u32), _vp]
 _lib.hccs_forward_static_scratch.restype = ctypes.c_int
+
+
+class _CalibGrid(ctypes.Structure):
+    _fields_ = [(k, _i32) for k in ("D_lo", "D_hi", "D_step", "S_lo", "S_hi", "S_step", "B_step")]
+
+
+_lib.hccs_calibrate.argtypes = [_vp, _i32, _i32, _i32, _i32, ctypes.c_double, ctypes.POINTER(_CalibGrid), _vp, _vp, _vp]
+_lib.hccs_calibrate.restype = ctypes.c_int
+
+
+def hccs_calibrate(logits, alpha: float, grid, stream=None):
+    """Grid-scan calibration of every head on device logits [B,H,Lq,Lk]; grid = (D_lo, D_hi, D_step,
+    S_lo, S_hi, S_step, B_step).  Returns (theta int32 [H,3], kl float64 [H])."""
+    B, H, Lq, Lk = logits.shape
+    _check_tensor(logits, "logits", 1)
+    g = _CalibGrid(*[int(v) for v in grid])
+    best = np.zeros((H, 3), dtype=np.int32)
+    kl = np.zeros(H, dtype=np.float64)
+    st = _lib.hccs_calibrate(_ptr(logits), B, H, Lq, Lk, float(alpha), ctypes.byref(g),
+                             best.ctypes.data_as(_vp), kl.ctypes.data_as(_vp), _stream_ptr(stream))
+    if st != HCCS_OK:
+        raise HccsError(st, "hccs_calibrate")
+    return best, kl
 
 
 def hccs_status_string(status: int) -> str:
