@@ -188,7 +188,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     __shared__ int part_max[4][kTile], part_sum[4][kTile];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nblk = a.L / kTile;                         // key blocks (and query tiles) per head
+    const int nblk = (a.L + kTile - 1) / kTile;           // key blocks (and query tiles) per head
+    const bool causal = (a.flags & HCCS_CAUSAL) != 0;
     volatile int *abortp = &abort_flag;
 
     // shared-memory carve-up (1024-byte aligned: required by the swizzled layouts)
@@ -241,7 +242,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // fetched while the previous tile is still in its softmax passes.
             auto prefetch = [&](int tile) {
                 const int bh = tile / nblk, qt = tile % nblk;
-                const int kblocks = CAUSAL ? qt + 1 : nblk;
+                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
                 mbar_expect_tx(smem_u32(&bars.q_full), kTileBytes);
                 tma_load_2d(s_q, &map_q, 0, bh * a.L + qt * kTile, smem_u32(&bars.q_full));
                 for (int kb = 0; kb < min(2, kblocks); ++kb) {
@@ -268,7 +269,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if ((int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int bh = tile / nblk, qt = tile % nblk;
-                const int kblocks = CAUSAL ? qt + 1 : nblk;
+                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
                 ok = mbar_wait(smem_u32(&bars.q_full), q_uses++ & 1, abortp, a.status);
                 for (int kb = 0; ok && kb < min(2, kblocks); ++kb) mma_qk(kb);
                 // the other K blocks land where the previous tile's V sits: wait for its last MMA
@@ -323,11 +324,13 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int bh = tile / nblk, qt = tile % nblk;
             const int head = bh % a.H;
             const int q0 = qt * kTile;
-            const int kblocks = CAUSAL ? qt + 1 : nblk;
+            const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
             const HeadEntry th = a.table[head];
             const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head);   // host-prepared constants
             const float out_scale = __int_as_float(a.requant_mult[8 * head + 4]);
-            const int nv = CAUSAL ? min(q0 + t + 1, a.L) : a.L;  // valid keys of this row
+            // valid keys of this row: all L of them, or the causal prefix (keys at and beyond L exist
+            // only as padding of the last block when L is no multiple of 128)
+            const int nv = (CAUSAL && causal) ? min(q0 + t + 1, a.L) : a.L;
 
             // the previous tile's O rows were staged in the panel: their bulk copies must have
             // read them before the panel is written again
@@ -516,7 +519,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             }
             if (tid == 0) leave_flag = *abortp;                   // one reader, so that all row threads agree
             asm volatile("bar.sync 1, 512;" ::: "memory");
-            if (ok && grp == 0) {
+            if (ok && grp == 0 && q0 + t < a.L) {
                 int32_t *o_row = (int32_t *)a.O + ((int64_t)bh * a.L + q0 + t) * kD;
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(o_row),
                              "r"(s_p + t * 272)
@@ -574,8 +577,8 @@ bool make_tile_map(CUtensorMap *map, const void *ptr, uint64_t rows) {
 template <bool CLB, bool CAUSAL>
 cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const FusedArgs &a,
                            cudaStream_t st) {
-    const int nblk = a.L / kTile;
-    size_t panel = (size_t)kTile * a.L;
+    const int nblk = (a.L + kTile - 1) / kTile;
+    size_t panel = (size_t)kTile * nblk * kTile;
     if (panel < (size_t)kTile * 272) panel = (size_t)kTile * 272;     // the O staging rows reuse the panel
     const size_t smem = 1024 + 3 * (size_t)kTileBytes + (size_t)nblk * kTileBytes + panel;
     auto kernel = fused_attention_kernel<CLB, CAUSAL>;
@@ -593,7 +596,7 @@ cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const C
 }  // namespace
 
 bool fused_shape_supported(int32_t L, int32_t d) {
-    return d == kD && L >= kTile && L <= kTile * kMaxBlocks && L % kTile == 0;
+    return d == kD && L >= 1 && L <= kTile * kMaxBlocks;
 }
 
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches) {
@@ -602,7 +605,8 @@ cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *laun
     if (!make_tile_map(&mq, a.Q, rows) || !make_tile_map(&mk, a.K, rows) || !make_tile_map(&mv, a.V, rows))
         return cudaErrorInvalidValue;
     cudaError_t e;
-    const bool clb = (a.flags & HCCS_RECIP_CLB) != 0, causal = (a.flags & HCCS_CAUSAL) != 0;
+    // the masked instantiation also serves L that is no multiple of 128 (padding keys in the last block)
+    const bool clb = (a.flags & HCCS_RECIP_CLB) != 0, causal = (a.flags & HCCS_CAUSAL) != 0 || a.L % kTile != 0;
     if (!clb && !causal) e = launch_variant<false, false>(mq, mk, mv, a, stream);
     else if (clb && !causal) e = launch_variant<true, false>(mq, mk, mv, a, stream);
     else if (!clb && causal) e = launch_variant<false, true>(mq, mk, mv, a, stream);

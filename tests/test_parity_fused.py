@@ -26,7 +26,7 @@ def _rand_qkv(rng, shape, lo=-64, hi=64):
     return tuple(rng.integers(lo, hi, size=shape, dtype=np.int8) for _ in range(3))
 
 
-@pytest.mark.parametrize("L", [128, 256, 640, 1024])
+@pytest.mark.parametrize("L", [1, 37, 128, 200, 256, 640, 1000, 1024])
 @pytest.mark.parametrize("flags", [0, 2, 4, 6])
 def test_small_heads(hccs, oracle, L, flags):
     rng = np.random.default_rng(1000 + L + flags)
@@ -74,7 +74,7 @@ def test_unsupported_shapes_are_refused(hccs):
     import torch
     ctx = hccs.Context(0)
     ctx.hccs_params_upload([(31, 1, 20)] * 2, 1024)
-    for L, d in ((100, 64), (128, 32), (2048, 64)):
+    for L, d in ((128, 32), (2048, 64), (1040, 64)):
         q = torch.zeros((1, 2, L, d), dtype=torch.int8, device="cuda")
         o = torch.zeros((1, 2, L, d), dtype=torch.int32, device="cuda")
         with pytest.raises(hccs.HccsError) as ei:
