@@ -45,7 +45,10 @@ constexpr int kTile = 128;                // queries per CTA, keys per block
 constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
 constexpr int kPanelBlockBytes = kTile * 128;   // 16 KB: 128 rows x 128 keys of the panel
 constexpr int kMaxBlocks = 8;             // L <= 1024
-constexpr uint32_t kTmemCols = 512;       // S0 [0,128)  S1 [128,256)  O [256,320)
+constexpr uint32_t kTmemCols = 512;       // S0 [0,128)  S1 [128,256)  S2 [256,384)  O [384,448)
+constexpr int kSBufs = 3;                 // S blocks in flight between the tensor core and the row warps
+constexpr uint32_t kTmemO = 384;
+constexpr uint32_t kOBoxBytes = 128 * 128; // one staged box of the output tile: 128 rows x 32 int32 columns
 constexpr long long kWaitCycles = 2000000000ll;
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -112,6 +115,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+// Tiled store of one shared-memory box to a 3-D tensor (rows past the tensor's extent are dropped).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int x, int y, int z, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map),
+                 "r"(x), "r"(y), "r"(z), "r"(src)
+                 : "memory");
+}
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
@@ -171,8 +180,8 @@ struct FusedSmemBarriers {
     uint64_t k_full[kMaxBlocks];
     uint64_t k_done;        // every MMA of the first contraction has finished reading K
     uint64_t v_full;
-    uint64_t s_full[2];
-    uint64_t s_free[2];
+    uint64_t s_full[kSBufs];
+    uint64_t s_free[kSBufs];
     uint64_t p_ready[kMaxBlocks];   // block kb of the probability panel is complete
     uint64_t o_full;
 };
@@ -180,7 +189,8 @@ struct FusedSmemBarriers {
 template <bool CLB, bool CAUSAL>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                       const __grid_constant__ CUtensorMap map_v, FusedArgs a, int num_tiles) {
+                       const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                       FusedArgs a, int num_tiles) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) FusedSmemBarriers bars;
     __shared__ uint32_t tmem_base_slot;
@@ -191,6 +201,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     const int nblk = (a.L + kTile - 1) / kTile;           // key blocks (and query tiles) per head
     const bool causal = (a.flags & HCCS_CAUSAL) != 0;
     volatile int *abortp = &abort_flag;
+    const bool two_rounds = a.requant_shift <= 24;        // see the row warps' scan flow
 
     // shared-memory carve-up (1024-byte aligned: required by the swizzled layouts)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -208,7 +219,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.k_full[i]), 1);
         mbar_init(smem_u32(&bars.k_done), 1);
         mbar_init(smem_u32(&bars.v_full), 1);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kSBufs; ++i) {
             mbar_init(smem_u32(&bars.s_full[i]), 1);
             mbar_init(smem_u32(&bars.s_free[i]), kRowThreads);
         }
@@ -237,7 +248,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             bool ok = true;
             uint32_t q_uses = 0, kdone_uses = 0, v_uses = 0, o_uses = 0;
             uint32_t k_par = 0, p_par = 0;               // bit kb = parity of the next use of k_full[kb] / p_ready[kb]
-            uint32_t s_uses[2] = {0, 0};
+            uint32_t s_buf = 0, s_cyc = 0;               // next S buffer and how often each was used so far
             // Q and the first two K blocks of a tile go to buffers of their own, so they can be
             // fetched while the previous tile is still in its softmax passes.
             auto prefetch = [&](int tile) {
@@ -250,13 +261,17 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
             };
-            auto mma_qk = [&](int kb) {                  // S[kb & 1] = Q . K_kb^T, two k-steps of 32 over d = 64
-                const int sb = kb & 1;
-                if (s_uses[sb] > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (s_uses[sb] - 1) & 1, abortp, a.status);
-                if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
+            // S[next buffer] = Q . K_kb^T, two k-steps of 32 over d = 64; the first use of a K block in a
+            // tile waits for its copy
+            auto mma_qk = [&](int kb, bool first_use) {
+                const uint32_t sb = s_buf;
+                if (s_cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (s_cyc - 1) & 1, abortp, a.status);
+                if (ok && first_use) {
+                    ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
+                    k_par ^= 1u << kb;
+                }
                 if (!ok) return;
-                k_par ^= 1u << kb;
-                ++s_uses[sb];
+                if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
                 tcgen05_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 2; ++ks) {
@@ -271,7 +286,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 const int bh = tile / nblk, qt = tile % nblk;
                 const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
                 ok = mbar_wait(smem_u32(&bars.q_full), q_uses++ & 1, abortp, a.status);
-                for (int kb = 0; ok && kb < min(2, kblocks); ++kb) mma_qk(kb);
+                for (int kb = 0; ok && kb < min(2, kblocks); ++kb) mma_qk(kb, true);
                 // the other K blocks land where the previous tile's V sits: wait for its last MMA
                 if (ok && it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (o_uses - 1) & 1, abortp, a.status);
                 if (!ok) break;
@@ -279,7 +294,11 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
                     tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
-                for (int kb = 2; ok && kb < kblocks; ++kb) mma_qk(kb);
+                for (int kb = 2; ok && kb < kblocks; ++kb) mma_qk(kb, true);
+                // the scan flow of the row warps reads every S block twice: once for the row maximum,
+                // once to requantise
+                if (two_rounds)
+                    for (int kb = 0; ok && kb < kblocks; ++kb) mma_qk(kb, false);
                 if (!ok) break;
                 tcgen05_commit(smem_u32(&bars.k_done));
                 ok = mbar_wait(smem_u32(&bars.k_done), kdone_uses++ & 1, abortp, a.status);
@@ -302,7 +321,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
                         const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
-                        tcgen05_mma_i8(tmem + 256, da, db, kIdescPV, (kb | ks) != 0);
+                        tcgen05_mma_i8(tmem + kTmemO, da, db, kIdescPV, (kb | ks) != 0);
                     }
                 }
                 if (!ok) break;
@@ -317,7 +336,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint8_t *row_base = panel + (t >> 3) * 1024 + (t & 7) * 128;
         const int swz = t & 7;
-        uint32_t sfull_uses[2] = {0, 0};                     // uses of s_full[0], s_full[1] by this thread
+        uint32_t s_buf = 0, s_cyc = 0;                       // S buffer of the next block and its use count
         bool ok = true;
 
         for (int tile = blockIdx.x, it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
@@ -335,122 +354,173 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // the previous tile's O rows were staged in the panel: their bulk copies must have
             // read them before the panel is written again
             if (it > 0) {
-                if (grp == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 asm volatile("bar.sync 1, 512;" ::: "memory");
             }
 
-            // ---- phase 1: requantise S into the panel and track the row maximum.
-            // x = clamp(floor((acc*M + R) / 2^sh), -128, 127) with R = 2^(sh-1).  The map is monotone
-            // and M < 2^(sh-1) makes its steps smaller than one, so clamping acc to [lo, hi] -- the
-            // accumulators that land exactly on -128 and 127 -- gives the same result with no later
-            // clamp.  With y = clamp(acc - lo, 0, hi - lo) (one instruction) and k = 24 - sh,
-            // t = y*(M << k) + ((lo*M + R) << k) lies in [-2^31, 2^31) and x is its top byte: one 32-bit
-            // multiply-add per logit, no shift, and the bytes are picked up by the packing PRMTs.
-            // The four constants come from the host, per head.  Shifts above 24 take the 64-bit
-            // multiply instead.
+            // ---- phases 1 and 2: the panel receives the closeness r = max(x + (D - m), 0) of every
+            // logit x = clamp(floor((acc*M + R) / 2^sh), -128, 127), R = 2^(sh-1), and the row gets m and
+            // the sum of r.
+            //
+            // Scan flow (shifts up to 24).  The requantisation is monotone, so m is the image of the
+            // largest accumulator: a first round over the S blocks only takes that maximum, and the
+            // control thread then issues the first contraction again.  In the second round, with
+            // t = m - D, every accumulator is clamped to [lo_t, hi] -- lo_t the smallest accumulator
+            // whose logit reaches max(t, -128), hi the largest one that gives 127 -- which performs the
+            // clamp of x and the clip of the distance at once (M < 2^(sh-1) makes the steps of the map
+            // smaller than one).  With y = clamp(acc - lo_t, 0, hi - lo_t) (one instruction) and
+            // k = 24 - sh, y*(M << k) + (((lo_t*M + R) << k) - (t << 24)) lies in [0, 2^31) and r is
+            // its top byte: one 32-bit multiply-add per logit, the bytes picked up by the packing
+            // PRMTs, their sum by one dot-product instruction per word.  Keys outside the mask get
+            // r = 0, so Z needs no correction.
+            //
+            // Shifts above 24 take the 64-bit multiply and keep the logits in the panel for a
+            // separate closeness pass.
             int xmax = -128;
-            if (a.requant_shift <= 24) {
+            uint32_t rsum = 0;
+            int cm = 0;
+            if (two_rounds) {
                 const uint32_t mk = (uint32_t)rq.x, ck = (uint32_t)rq.y;
                 const int neg_lo = rq.z, span = rq.w;
-                int ymax = 0;
+                int amax = -(1 << 30);
                 for (int kb = 0; ok && kb < kblocks; ++kb) {
-                    const int sb = kb & 1;
-                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), sfull_uses[sb] & 1, abortp, a.status);
+                    const uint32_t sb = s_buf;
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
                     if (!ok) break;
-                    ++sfull_uses[sb];
+                    if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
                     tcgen05_fence_after();
-                    uint8_t *blk = row_base + kb * kPanelBlockBytes;
-                    {
-                        const int j = grp;
-                        uint32_t acc[32];
-                        tmem_ld32(tmem + lane_addr + sb * 128 + j * 32, acc);
-                        uint32_t w[8];
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+                    const int c0 = kb * kTile + grp * 32;
+                    if (CAUSAL && c0 + 32 > nv) {
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            uint32_t tt[4];
-                            int y[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                y[e] = __viaddmin_s32_relu((int)acc[4 * g + e], neg_lo, span);
-                                tt[e] = (uint32_t)y[e] * mk + ck;
-                                if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) { tt[e] = 0x80000000u; y[e] = 0; }
-                            }
-                            w[g] = prmt(prmt(tt[0], tt[1], 0x0073u), prmt(tt[2], tt[3], 0x0073u), 0x5410u);
-                            ymax = __vimax3_s32(__vimax3_s32(ymax, y[0], y[1]), y[2], y[3]);
-                        }
-                        *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                        *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                        for (int e = 0; e < 32; ++e)
+                            if (c0 + e >= nv) acc[e] = (uint32_t)(-(1 << 30));
                     }
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) amax = __vimax3_s32(amax, (int)acc[e], (int)acc[e + 1]);
                     tcgen05_fence_before();
                     mbar_arrive(smem_u32(&bars.s_free[sb]));
                 }
-                xmax = (int)((uint32_t)ymax * mk + ck) >> 24;
+                xmax = (int)((uint32_t)__viaddmin_s32_relu(amax, neg_lo, span) * mk + ck) >> 24;
+                part_max[grp][t] = xmax;
+                asm volatile("bar.sync 1, 512;" ::: "memory");        // the row threads only
+                xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
+                cm = th.D - xmax;
+
+                // lo_t = clamp(ceil((t*2^sh - R) / M), lo, hi): two single-precision estimates of the
+                // quotient (the second on the remainder of the first, which leaves at most one unit
+                // of error) and integer corrections
+                const int sh = a.requant_shift, kk = 24 - sh;
+                const int M = (int)(mk >> kk), lo = -neg_lo, hi = lo + span;
+                const int64_t R = (int64_t)1 << (sh - 1);
+                const int64_t want = (int64_t)(-cm) * ((int64_t)1 << sh);       // t * 2^sh
+                int lo_t = lo;
+                if (M > 0) {
+                    const float inv_m = 1.0f / (float)M;
+                    const int64_t num = want - R;
+                    int q = (int)fminf(fmaxf(floorf((float)num * inv_m), (float)(lo - 1)), (float)(hi + 1));
+                    q += (int)fminf(fmaxf(floorf((float)(num - (int64_t)q * M) * inv_m), -8388608.0f), 8388608.0f);
+                    q = min(max(q, lo - 4), hi + 4);
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+                        if ((int64_t)q * M < num) ++q;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+                        if ((int64_t)(q - 1) * M >= num) --q;
+                    lo_t = min(max(q, lo), hi);
+                }
+                const int neg_lo_t = -lo_t, span_t = hi - lo_t;
+                const uint32_t ck_t =
+                    ((uint32_t)((int64_t)lo_t * M + R) << kk) - ((uint32_t)(-cm) << 24);
+                for (int kb = 0; ok && kb < kblocks; ++kb) {
+                    const uint32_t sb = s_buf;
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
+                    if (!ok) break;
+                    if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
+                    tcgen05_fence_after();
+                    uint8_t *blk = row_base + kb * kPanelBlockBytes;
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+                    uint32_t w[8];
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        uint32_t tt[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            tt[e] = (uint32_t)__viaddmin_s32_relu((int)acc[4 * g + e], neg_lo_t, span_t) * mk + ck_t;
+                            if (CAUSAL && kb * kTile + grp * 32 + 4 * g + e >= nv) tt[e] = 0u;
+                        }
+                        w[g] = prmt(prmt(tt[0], tt[1], 0x0073u), prmt(tt[2], tt[3], 0x0073u), 0x5410u);
+                        rsum = __dp4a(w[g], 0x01010101u, rsum);
+                    }
+                    *reinterpret_cast<uint4 *>(blk + (((2 * grp) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(blk + (((2 * grp + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                    tcgen05_fence_before();
+                    mbar_arrive(smem_u32(&bars.s_free[sb]));
+                }
             } else {
                 const int32_t mult_hi = rq.x << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
                 for (int kb = 0; ok && kb < kblocks; ++kb) {
-                    const int sb = kb & 1;
-                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), sfull_uses[sb] & 1, abortp, a.status);
+                    const uint32_t sb = s_buf;
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
                     if (!ok) break;
-                    ++sfull_uses[sb];
+                    if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
                     tcgen05_fence_after();
                     uint8_t *blk = row_base + kb * kPanelBlockBytes;
-                    {
-                        const int j = grp;
-                        uint32_t acc[32];
-                        tmem_ld32(tmem + lane_addr + sb * 128 + j * 32, acc);
-                        uint32_t w[8];
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+                    uint32_t w[8];
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            int32_t x[4];
+                    for (int g = 0; g < 8; ++g) {
+                        int32_t x[4];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
-                                if (CAUSAL && kb * kTile + j * 32 + 4 * g + e >= nv) x[e] = -128;
-                            }
-                            w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
-                            xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
+                        for (int e = 0; e < 4; ++e) {
+                            x[e] = (int32_t)(mad_wide_s32((int32_t)acc[4 * g + e], mult_hi, (int64_t)1 << 31) >> 32);
+                            if (CAUSAL && kb * kTile + grp * 32 + 4 * g + e >= nv) x[e] = -128;
                         }
-                        *reinterpret_cast<uint4 *>(blk + (((2 * j) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                        *reinterpret_cast<uint4 *>(blk + (((2 * j + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                        w[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
+                        xmax = max(xmax, max(max(x[0], x[1]), max(x[2], x[3])));
                     }
+                    *reinterpret_cast<uint4 *>(blk + (((2 * grp) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(blk + (((2 * grp + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
                     tcgen05_fence_before();
                     mbar_arrive(smem_u32(&bars.s_free[sb]));
                 }
-            }
-            xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
-            part_max[grp][t] = xmax;
-            asm volatile("bar.sync 1, 512;" ::: "memory");        // the row threads only
-            xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
+                xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
+                part_max[grp][t] = xmax;
+                asm volatile("bar.sync 1, 512;" ::: "memory");
+                xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
+                cm = th.D - xmax;
 
-            // ---- phase 2: closeness r = max(x + (D - m), 0), stored back in place of the logit; its sum
-            const int cm = th.D - xmax;
-            const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
-            uint32_t rsum = 0;
-            for (int kb = 0; kb < kblocks; ++kb) {
-                uint8_t *blk = row_base + kb * kPanelBlockBytes;
-                uint4 v[2];
+                // closeness pass over the stored logits, in place; masked keys were stored as -128 and
+                // contribute max(cm - 128, 0) each, which is taken out of the row's sum below
+                const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    uint8_t *blk = row_base + kb * kPanelBlockBytes;
+                    uint4 v[2];
 #pragma unroll
-                for (int c = 0; c < 2; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((2 * grp + c) ^ swz) << 4));
+                    for (int c = 0; c < 2; ++c) v[c] = *reinterpret_cast<const uint4 *>(blk + (((2 * grp + c) ^ swz) << 4));
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-                    uint32_t s2 = 0;
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                        uint32_t s2 = 0;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
-                        const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
-                        s2 += ev + od;
-                        w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
+                        for (int k = 0; k < 4; ++k) {
+                            const uint32_t ev = __viaddmax_s16x2(prmt(w[k], 0, 0xA280u), c2, 0u);
+                            const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
+                            s2 += ev + od;
+                            w[k] = prmt(ev, od, 0x6240u);             // r bytes back in key order
+                        }
+                        rsum += (s2 & 0xffffu) + (s2 >> 16);
+                        *reinterpret_cast<uint4 *>(blk + (((2 * grp + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
-                    rsum += (s2 & 0xffffu) + (s2 >> 16);
-                    *reinterpret_cast<uint4 *>(blk + (((2 * grp + c) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
             part_sum[grp][t] = (int)rsum;
             asm volatile("bar.sync 1, 512;" ::: "memory");
-            const int rs_all = part_sum[0][t] + part_sum[1][t] + part_sum[2][t] + part_sum[3][t];
-            const int masked = kblocks * kTile - nv;                         // keys stored as -128
-            const int rs = rs_all - masked * max(cm - 128, 0);
+            int rs = part_sum[0][t] + part_sum[1][t] + part_sum[2][t] + part_sum[3][t];
+            if (!two_rounds) rs -= (kblocks * kTile - nv) * max(cm - 128, 0);
             const int F = th.B - th.S * th.D;
             const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
             const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
@@ -498,38 +568,38 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // ---- phase 4: O out of tensor memory.  A thread holds 16 columns of its row; writing them
             // straight to global memory would cost one memory transaction per lane (rows are 256 bytes
             // apart), so the tile goes through shared memory (the panel, free once the second
-            // contraction is complete; rows padded to 272 bytes to spread the banks) and leaves as one
-            // 256-byte bulk copy per row.
+            // contraction is complete) as two boxes of 128 rows x 32 columns in the 128-byte swizzled
+            // layout -- which also spreads a warp's 16-byte stores over all banks -- and one thread
+            // sends both boxes off as tiled bulk stores; rows beyond L fall outside the tensor map
+            // and are dropped.
             if (ok) ok = mbar_wait(smem_u32(&bars.o_full), it & 1, abortp, a.status);
             if (ok) {
                 tcgen05_fence_after();
                 uint32_t acc[16];
-                tmem_ld16(tmem + lane_addr + 256 + grp * 16, acc);
+                tmem_ld16(tmem + lane_addr + kTmemO + grp * 16, acc);
                 if (a.out_f32) {                                  // optional dequantised view of O
 #pragma unroll
                     for (int g = 0; g < 16; ++g) acc[g] = __float_as_uint(__int2float_rn((int)acc[g]) * out_scale);
                 }
-                uint8_t *o_stage = panel + t * 272;
+                uint8_t *o_stage = panel + (grp >> 1) * kOBoxBytes + t * 128;
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
-                    *reinterpret_cast<uint4 *>(o_stage + grp * 64 + g * 16) =
+                    *reinterpret_cast<uint4 *>(o_stage + ((((grp & 1) * 4 + g) ^ swz) << 4)) =
                         make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
                 tcgen05_fence_before();
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             if (tid == 0) leave_flag = *abortp;                   // one reader, so that all row threads agree
             asm volatile("bar.sync 1, 512;" ::: "memory");
-            if (ok && grp == 0 && q0 + t < a.L) {
-                int32_t *o_row = (int32_t *)a.O + ((int64_t)bh * a.L + q0 + t) * kD;
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(o_row),
-                             "r"(s_p + t * 272)
-                             : "memory");
+            if (tid == 0 && !*(volatile int *)&leave_flag) {
+                tma_store_3d(&map_o, 0, q0, bh, s_p);
+                tma_store_3d(&map_o, 32, q0, bh, s_p + kOBoxBytes);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
             // leave the loop together (the flag was sampled once, before the barrier above)
             if (*(volatile int *)&leave_flag) break;
         }
-        if (grp == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem must outlive the reads
+        if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem must outlive the reads
     }
 
     // ===================================================== common exit: free the tensor memory
@@ -574,12 +644,26 @@ bool make_tile_map(CUtensorMap *map, const void *ptr, uint64_t rows) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// O as [B*H][L][64] 32-bit words, boxes of 128 rows x 32 words, 128-byte swizzle.  Three dimensions, so
+// that a tile of the last, partial row block of a head stops at the head's end.
+bool make_output_map(CUtensorMap *map, const void *ptr, uint64_t heads, uint64_t L) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)L, (cuuint64_t)heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 4, (cuuint64_t)kD * 4 * L};
+    const cuuint32_t box[3] = {32, (cuuint32_t)kTile, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool CLB, bool CAUSAL>
-cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const FusedArgs &a,
-                           cudaStream_t st) {
+cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mo,
+                           const FusedArgs &a, cudaStream_t st) {
     const int nblk = (a.L + kTile - 1) / kTile;
     size_t panel = (size_t)kTile * nblk * kTile;
-    if (panel < (size_t)kTile * 272) panel = (size_t)kTile * 272;     // the O staging rows reuse the panel
+    if (panel < 2 * (size_t)kOBoxBytes) panel = 2 * (size_t)kOBoxBytes;   // the staged O boxes reuse the panel
     const size_t smem = 1024 + 3 * (size_t)kTileBytes + (size_t)nblk * kTileBytes + panel;
     auto kernel = fused_attention_kernel<CLB, CAUSAL>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -589,7 +673,7 @@ cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const C
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const unsigned blocks = (unsigned)(tiles < sms ? tiles : sms);      // persistent: one CTA per SM
-    kernel<<<blocks, kThreads, smem, st>>>(mq, mk, mv, a, (int)tiles);
+    kernel<<<blocks, kThreads, smem, st>>>(mq, mk, mv, mo, a, (int)tiles);
     return cudaGetLastError();
 }
 
@@ -600,17 +684,18 @@ bool fused_shape_supported(int32_t L, int32_t d) {
 }
 
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches) {
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     const uint64_t rows = (uint64_t)a.B * a.H * a.L;
-    if (!make_tile_map(&mq, a.Q, rows) || !make_tile_map(&mk, a.K, rows) || !make_tile_map(&mv, a.V, rows))
+    if (!make_tile_map(&mq, a.Q, rows) || !make_tile_map(&mk, a.K, rows) || !make_tile_map(&mv, a.V, rows) ||
+        !make_output_map(&mo, a.O, (uint64_t)a.B * a.H, (uint64_t)a.L))
         return cudaErrorInvalidValue;
     cudaError_t e;
     // the masked instantiation also serves L that is no multiple of 128 (padding keys in the last block)
     const bool clb = (a.flags & HCCS_RECIP_CLB) != 0, causal = (a.flags & HCCS_CAUSAL) != 0 || a.L % kTile != 0;
-    if (!clb && !causal) e = launch_variant<false, false>(mq, mk, mv, a, stream);
-    else if (clb && !causal) e = launch_variant<true, false>(mq, mk, mv, a, stream);
-    else if (!clb && causal) e = launch_variant<false, true>(mq, mk, mv, a, stream);
-    else e = launch_variant<true, true>(mq, mk, mv, a, stream);
+    if (!clb && !causal) e = launch_variant<false, false>(mq, mk, mv, mo, a, stream);
+    else if (clb && !causal) e = launch_variant<true, false>(mq, mk, mv, mo, a, stream);
+    else if (!clb && causal) e = launch_variant<false, true>(mq, mk, mv, mo, a, stream);
+    else e = launch_variant<true, true>(mq, mk, mv, mo, a, stream);
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }

@@ -55,6 +55,22 @@ def test_full_range_int8_and_saturating_requant(hccs, oracle):
         assert_same(got, want, f"fused full-range sh={sh} os={out_shift}")
 
 
+@pytest.mark.parametrize("sh,mults", [(24, [0, 1, 8191]), (14, [8191, 100, 3]), (8, [127, 1, 64]),
+                                      (2, [1, 0, 1]), (25, [8191, 0, 1])])
+@pytest.mark.parametrize("flags", [0, 4])
+def test_requantisation_corner_cases(hccs, oracle, sh, mults, flags):
+    """Multipliers 0 and 1, the largest multiplier each shift admits, tiny and large shifts (both
+    requantisation flows of the kernel), on a ragged length with full-range int8 operands."""
+    rng = np.random.default_rng(77 + sh + flags)
+    Bt, H, L, d = 2, 3, 200, 64
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
+    theta = hccs.workloads.sample_theta(rng, H, L)
+    mult = np.array(mults, dtype=np.int32)
+    got = _run(hccs, Q, K, V, theta, mult, sh, L, flags)
+    want = oracle.attention(Q, K, V, mult, sh, theta, oracle_mode(oracle, flags), threads=8)
+    assert_same(got, want, f"fused requant sh={sh} mult={mults} flags={flags}")
+
+
 def test_config5_sampled_heads(hccs, oracle):
     """The benchmark's fused workload at full size; the oracle recomputes a sample of heads."""
     wl = hccs.workloads.make_config(5)
