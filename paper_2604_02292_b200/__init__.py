@@ -8,6 +8,7 @@ import importlib
 from . import workloads  # noqa: F401
 
 __all__ = ["workloads"]
+_SUBMODULES = ("build", "binding", "calibrate_report")
 
 
 def __getattr__(name):
@@ -15,6 +16,8 @@ def __getattr__(name):
     # the compiled library; a missing library is an ImportError, never a fallback.
     if name.startswith("__"):
         raise AttributeError(name)
+    if name in _SUBMODULES:                  # `from package import build` must work before the library exists
+        return importlib.import_module(__name__ + "." + name)
     binding = importlib.import_module(__name__ + ".binding")
     try:
         return getattr(binding, name)
