@@ -17,13 +17,16 @@
 //   * V is used as stored ([key][64], keys outermost): that is exactly the MN-major, 64-byte
 //     swizzled B operand, so no transposition is needed.
 //
-// Warp roles (544 threads): warps 0-15 are row warps, four threads per query row (threads t,
+// Warp roles (608 threads): warps 0-15 are row warps, four threads per query row (threads t,
 // t + 128, t + 256, t + 384 own row t mod 128; TMEM lane quarter = warp index mod 4): bits 7-8
 // of the thread index select which 32 of the 128 keys of every block the thread handles, so all
-// row threads work on the same block while the tensor core fills the other S buffer.
+// row threads work on the same block while the tensor core fills the other S buffers.
 // The four exchange their partial row max and row sum through shared memory; the many warps are
-// what hides the latency of the dependent integer chains.  Warp 16 lane 0 issues every TMA copy
-// and every MMA.  All mbarrier waits are bounded; a wait that runs
+// what hides the latency of the dependent integer chains.  Three more warps each run one
+// single-lane role on a scheduler of their own: warp 16 issues every TMA load, warp 17 the first
+// contraction, warp 18 the second (one thread doing all three fell behind the row warps: its
+// serial chain of waits, descriptor arithmetic and issues cost several hundred cycles per block).
+// All mbarrier waits are bounded; a wait that runs
 // out sets STATUS_FUSED_TIMEOUT, raises an abort flag that every other wait observes, and the CTA
 // leaves through the common exit, which frees its tensor memory.  No clusters, no multicast.
 #include <cuda.h>
@@ -38,8 +41,8 @@ namespace hccs {
 namespace {
 
 constexpr int kRowThreads = 512;           // four per query row
-constexpr int kThreads = 544;
-constexpr int kCtlWarp = 16;
+constexpr int kThreads = 608;            // 16 row warps and three single-lane role warps
+constexpr int kTmaWarp = 16, kQkWarp = 17, kPvWarp = 18;
 constexpr int kD = 64;                    // head dimension (bytes per Q/K/V row)
 constexpr int kTile = 128;                // queries per CTA, keys per block
 constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
@@ -61,6 +64,11 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 __device__ __forceinline__ uint64_t mad_wide_u32(uint32_t a, uint32_t b, uint64_t c) {
     uint64_t d;
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t make_u64(uint32_t lo, uint32_t hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
     return d;
 }
 __device__ __forceinline__ int64_t mad_wide_s32(int32_t a, int32_t b, int64_t c) {
@@ -179,7 +187,7 @@ struct FusedSmemBarriers {
     uint64_t q_full;
     uint64_t k_full[kMaxBlocks];
     uint64_t k_done;        // every MMA of the first contraction has finished reading K
-    uint64_t v_full;
+    uint64_t v_full[kMaxBlocks];
     uint64_t s_full[kSBufs];
     uint64_t s_free[kSBufs];
     uint64_t p_ready[kMaxBlocks];   // block kb of the probability panel is complete
@@ -218,7 +226,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         mbar_init(smem_u32(&bars.q_full), 1);
         for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.k_full[i]), 1);
         mbar_init(smem_u32(&bars.k_done), 1);
-        mbar_init(smem_u32(&bars.v_full), 1);
+        for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.v_full[i]), 1);
         for (int i = 0; i < kSBufs; ++i) {
             mbar_init(smem_u32(&bars.s_full[i]), 1);
             mbar_init(smem_u32(&bars.s_free[i]), kRowThreads);
@@ -228,7 +236,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == kCtlWarp) {   // one warp allocates the tensor memory for the CTA
+    if (warp == kTmaWarp) {   // one warp allocates the tensor memory for the CTA
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(kTmemCols)
                      : "memory");
@@ -242,13 +250,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     // A CTA walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every mbarrier completes
     // one phase per use, so both sides count their uses (per barrier, because a causal tile uses
     // only its first qt + 1 key blocks) and wait on the parity of that count.
-    if (warp == kCtlWarp) {
-        // ===================================================== control thread: TMA + MMA issue
+    if (warp == kTmaWarp) {
+        // ===================================================== copy thread: every TMA load
         if (lane == 0) {
             bool ok = true;
-            uint32_t q_uses = 0, kdone_uses = 0, v_uses = 0, o_uses = 0;
-            uint32_t k_par = 0, p_par = 0;               // bit kb = parity of the next use of k_full[kb] / p_ready[kb]
-            uint32_t s_buf = 0, s_cyc = 0;               // next S buffer and how often each was used so far
             // Q and the first two K blocks of a tile go to buffers of their own, so they can be
             // fetched while the previous tile is still in its softmax passes.
             auto prefetch = [&](int tile) {
@@ -261,72 +266,101 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
             };
-            // S[next buffer] = Q . K_kb^T, two k-steps of 32 over d = 64; the first use of a K block in a
-            // tile waits for its copy
-            auto mma_qk = [&](int kb, bool first_use) {
-                const uint32_t sb = s_buf;
-                if (s_cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (s_cyc - 1) & 1, abortp, a.status);
-                if (ok && first_use) {
-                    ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
-                    k_par ^= 1u << kb;
-                }
-                if (!ok) return;
-                if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
-                tcgen05_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 2; ++ks) {
-                    const uint64_t da = smem_desc(s_q + ks * 32, 16, 512, kSwizzle64);
-                    const uint64_t db = smem_desc(k_slot(kb) + ks * 32, 16, 512, kSwizzle64);
-                    tcgen05_mma_i8(tmem + sb * 128, da, db, kIdescQK, ks);
-                }
-                tcgen05_commit(smem_u32(&bars.s_full[sb]));
-            };
             if ((int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int bh = tile / nblk, qt = tile % nblk;
                 const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
-                ok = mbar_wait(smem_u32(&bars.q_full), q_uses++ & 1, abortp, a.status);
-                for (int kb = 0; ok && kb < min(2, kblocks); ++kb) mma_qk(kb, true);
                 // the other K blocks land where the previous tile's V sits: wait for its last MMA
-                if (ok && it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (o_uses - 1) & 1, abortp, a.status);
+                if (it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (it - 1) & 1, abortp, a.status);
                 if (!ok) break;
                 for (int kb = 2; kb < kblocks; ++kb) {
                     mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
                     tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
-                for (int kb = 2; ok && kb < kblocks; ++kb) mma_qk(kb, true);
+                // V takes the K buffer once the first contraction has read the last K block; Q and
+                // the first K blocks of the next tile are fetched as well
+                ok = mbar_wait(smem_u32(&bars.k_done), it & 1, abortp, a.status);
+                if (!ok) break;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    mbar_expect_tx(smem_u32(&bars.v_full[kb]), kTileBytes);
+                    tma_load_2d(s_kv + kb * kTileBytes, &map_v, 0, bh * a.L + kb * kTile, smem_u32(&bars.v_full[kb]));
+                }
+                if (tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
+            }
+        }
+    } else if (warp == kQkWarp) {
+        // ===================================================== first contraction: S = Q . K^T, block by block
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t k_par = 0;                          // bit kb = parity of the next use of k_full[kb]
+            uint32_t s_buf = 0, s_cyc = 0;               // next S buffer and how often each was used so far
+            // descriptors differ only in the start address field (address >> 4): low word + offset
+            const uint64_t dq = smem_desc(s_q, 16, 512, kSwizzle64);
+            const uint64_t dk = smem_desc(s_kpre, 16, 512, kSwizzle64);
+            const uint32_t dq_lo = (uint32_t)dq, dq_hi = (uint32_t)(dq >> 32);
+            const uint32_t dk_lo = (uint32_t)dk, dk_hi = (uint32_t)(dk >> 32);
+            for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                const int qt = tile % nblk;
+                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+                ok = mbar_wait(smem_u32(&bars.q_full), it & 1, abortp, a.status);
                 // the scan flow of the row warps reads every S block twice: once for the row maximum,
                 // once to requantise
-                if (two_rounds)
-                    for (int kb = 0; ok && kb < kblocks; ++kb) mma_qk(kb, false);
+                for (int round = 0; ok && round < (two_rounds ? 2 : 1); ++round) {
+#pragma unroll
+                    for (int kb = 0; kb < kMaxBlocks; ++kb) {
+                        if (kb >= kblocks || !ok) break;
+                        const uint32_t sb = s_buf;
+                        if (s_cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (s_cyc - 1) & 1, abortp, a.status);
+                        if (ok && round == 0) {          // the first use of a K block waits for its copy
+                            ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
+                            k_par ^= 1u << kb;
+                        }
+                        if (!ok) break;
+                        if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
+                        tcgen05_fence_after();
+                        // K block kb sits (kb < 2 ? kb : kb + 2) tiles above the first prefetch slot;
+                        // two k-steps of 32 over d = 64
+                        const uint32_t koff = (uint32_t)((kb < 2 ? kb : kb + 2) * kTileBytes) >> 4;
+                        tcgen05_mma_i8(tmem + sb * 128, make_u64(dq_lo, dq_hi), make_u64(dk_lo + koff, dk_hi), kIdescQK, 0);
+                        tcgen05_mma_i8(tmem + sb * 128, make_u64(dq_lo + 2, dq_hi), make_u64(dk_lo + koff + 2, dk_hi), kIdescQK, 1);
+                        tcgen05_commit(smem_u32(&bars.s_full[sb]));
+                    }
+                }
                 if (!ok) break;
                 tcgen05_commit(smem_u32(&bars.k_done));
-                ok = mbar_wait(smem_u32(&bars.k_done), kdone_uses++ & 1, abortp, a.status);
-                if (!ok) break;
-                // ---- V takes the K buffer while the row warps run the softmax passes; Q and the
-                // first K blocks of the next tile are fetched as well
-                mbar_expect_tx(smem_u32(&bars.v_full), (uint32_t)kblocks * kTileBytes);
-                for (int kb = 0; kb < kblocks; ++kb)
-                    tma_load_2d(s_kv + kb * kTileBytes, &map_v, 0, bh * a.L + kb * kTile, smem_u32(&bars.v_full));
-                if (tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
-                ok = mbar_wait(smem_u32(&bars.v_full), v_uses++ & 1, abortp, a.status);
-                // ---- second contraction, block by block as the row warps finish the probabilities:
-                // four k-steps of 32 keys per block
-                for (int kb = 0; ok && kb < kblocks; ++kb) {
-                    ok = mbar_wait(smem_u32(&bars.p_ready[kb]), (p_par >> kb) & 1, abortp, a.status);
+            }
+        }
+    } else if (warp == kPvWarp) {
+        // ===================================================== second contraction: O += P_kb . V_kb as the
+        // row warps finish the probability blocks; four k-steps of 32 keys per block
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t p_par = 0;                          // bit kb = parity of the next use of p_ready[kb] and v_full[kb]
+            const uint64_t dp = smem_desc(s_p, 16, 1024, kSwizzle128);
+            const uint64_t dv = smem_desc(s_kv, 512, 512, kSwizzle64);
+            const uint32_t dp_lo = (uint32_t)dp, dp_hi = (uint32_t)(dp >> 32);
+            const uint32_t dv_lo = (uint32_t)dv, dv_hi = (uint32_t)(dv >> 32);
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int qt = tile % nblk;
+                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+#pragma unroll
+                for (int kb = 0; kb < kMaxBlocks; ++kb) {
+                    if (kb >= kblocks) break;
+                    ok = mbar_wait(smem_u32(&bars.v_full[kb]), (p_par >> kb) & 1, abortp, a.status);
+                    if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[kb]), (p_par >> kb) & 1, abortp, a.status);
                     if (!ok) break;
                     p_par ^= 1u << kb;
                     tcgen05_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t da = smem_desc(s_p + kb * kPanelBlockBytes + ks * 32, 16, 1024, kSwizzle128);
-                        const uint64_t db = smem_desc(s_kv + (kb * kTile + ks * 32) * kD, 512, 512, kSwizzle64);
-                        tcgen05_mma_i8(tmem + kTmemO, da, db, kIdescPV, (kb | ks) != 0);
+                        const uint32_t poff = (uint32_t)(kb * kPanelBlockBytes + ks * 32) >> 4;
+                        const uint32_t voff = (uint32_t)((kb * kTile + ks * 32) * kD) >> 4;
+                        tcgen05_mma_i8(tmem + kTmemO, make_u64(dp_lo + poff, dp_hi), make_u64(dv_lo + voff, dv_hi), kIdescPV,
+                                       (kb | ks) != 0);
                     }
                 }
                 if (!ok) break;
                 tcgen05_commit(smem_u32(&bars.o_full));
-                ++o_uses;
             }
         }
     } else {
@@ -353,7 +387,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 
             // the previous tile's O rows were staged in the panel: their bulk copies must have
             // read them before the panel is written again
-            if (it > 0) {
+            // (the scan flow first writes the panel after its first round, whose closing barrier serves)
+            if (it > 0 && !two_rounds) {
                 if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 asm volatile("bar.sync 1, 512;" ::: "memory");
             }
@@ -364,7 +399,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             //
             // Scan flow (shifts up to 24).  The requantisation is monotone, so m is the image of the
             // largest accumulator: a first round over the S blocks only takes that maximum, and the
-            // control thread then issues the first contraction again.  In the second round, with
+            // first contraction is then issued again.  In the second round, with
             // t = m - D, every accumulator is clamped to [lo_t, hi] -- lo_t the smallest accumulator
             // whose logit reaches max(t, -128), hi the largest one that gives 127 -- which performs the
             // clamp of x and the clip of the distance at once (M < 2^(sh-1) makes the steps of the map
@@ -404,6 +439,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 }
                 xmax = (int)((uint32_t)__viaddmin_s32_relu(amax, neg_lo, span) * mk + ck) >> 24;
                 part_max[grp][t] = xmax;
+                if (tid == 0 && it > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 asm volatile("bar.sync 1, 512;" ::: "memory");        // the row threads only
                 xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
                 cm = th.D - xmax;
@@ -604,7 +640,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 
     // ===================================================== common exit: free the tensor memory
     __syncthreads();
-    if (warp == kCtlWarp) {
+    if (warp == kTmaWarp) {
         tcgen05_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
