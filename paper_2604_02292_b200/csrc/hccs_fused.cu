@@ -17,15 +17,16 @@
 //   * V is used as stored ([key][64], keys outermost): that is exactly the MN-major, 64-byte
 //     swizzled B operand, so no transposition is needed.
 //
-// Warp roles (608 threads): warps 0-15 are row warps, four threads per query row (threads t,
+// Warp roles (640 threads): warps 0-15 are row warps, four threads per query row (threads t,
 // t + 128, t + 256, t + 384 own row t mod 128; TMEM lane quarter = warp index mod 4): bits 7-8
 // of the thread index select which 32 of the 128 keys of every block the thread handles, so all
 // row threads work on the same block while the tensor core fills the other S buffers.
 // The four exchange their partial row max and row sum through shared memory; the many warps are
-// what hides the latency of the dependent integer chains.  Three more warps each run one
-// single-lane role on a scheduler of their own: warp 16 issues every TMA load, warp 17 the first
-// contraction, warp 18 the second (one thread doing all three fell behind the row warps: its
-// serial chain of waits, descriptor arithmetic and issues cost several hundred cycles per block).
+// what hides the latency of the dependent integer chains.  Four more warps each run one
+// single-lane role on a scheduler of their own: warp 16 issues every TMA load, warps 17 and 19
+// the first contraction (alternate blocks), warp 18 the second (one thread doing it all fell
+// behind the row warps: its serial chain of waits, descriptor arithmetic and issues cost several
+// hundred cycles per block).
 // All mbarrier waits are bounded; a wait that runs
 // out sets STATUS_FUSED_TIMEOUT, raises an abort flag that every other wait observes, and the CTA
 // leaves through the common exit, which frees its tensor memory.  No clusters, no multicast.
@@ -41,8 +42,8 @@ namespace hccs {
 namespace {
 
 constexpr int kRowThreads = 512;           // four per query row
-constexpr int kThreads = 608;            // 16 row warps and three single-lane role warps
-constexpr int kTmaWarp = 16, kQkWarp = 17, kPvWarp = 18;
+constexpr int kThreads = 640;            // 16 row warps and four single-lane role warps
+constexpr int kTmaWarp = 16, kQkWarp = 17, kPvWarp = 18, kQk2Warp = 19;
 constexpr int kD = 64;                    // head dimension (bytes per Q/K/V row)
 constexpr int kTile = 128;                // queries per CTA, keys per block
 constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
@@ -225,7 +226,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         abort_flag = 0;
         mbar_init(smem_u32(&bars.q_full), 1);
         for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.k_full[i]), 1);
-        mbar_init(smem_u32(&bars.k_done), 1);
+        mbar_init(smem_u32(&bars.k_done), 2);
         for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.v_full[i]), 1);
         for (int i = 0; i < kSBufs; ++i) {
             mbar_init(smem_u32(&bars.s_full[i]), 1);
@@ -288,12 +289,16 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 if (tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
             }
         }
-    } else if (warp == kQkWarp) {
-        // ===================================================== first contraction: S = Q . K^T, block by block
+    } else if (warp == kQkWarp || warp == kQk2Warp) {
+        // ===================================================== first contraction: S = Q . K^T, block by block.
+        // Two issuers take the blocks alternately: what one thread spends per block (two waits, the
+        // descriptors, two MMAs, the commit) is more than the tensor core needs for it.
         if (lane == 0) {
+            const uint32_t me = warp == kQkWarp ? 0u : 1u;
             bool ok = true;
-            uint32_t k_par = 0;                          // bit kb = parity of the next use of k_full[kb]
-            uint32_t s_buf = 0, s_cyc = 0;               // next S buffer and how often each was used so far
+            uint32_t k_par = 0;                          // bit kb = parity of this tile's phase of k_full[kb]
+            uint32_t g = 0;                              // blocks issued so far by both issuers
+            uint32_t s_buf = 0, s_cyc = 0;               // = g % kSBufs, g / kSBufs: S buffer of block g and its use
             // descriptors differ only in the start address field (address >> 4): low word + offset
             const uint64_t dq = smem_desc(s_q, 16, 512, kSwizzle64);
             const uint64_t dk = smem_desc(s_kpre, 16, 512, kSwizzle64);
@@ -309,14 +314,16 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                     for (int kb = 0; kb < kMaxBlocks; ++kb) {
                         if (kb >= kblocks || !ok) break;
-                        const uint32_t sb = s_buf;
-                        if (s_cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (s_cyc - 1) & 1, abortp, a.status);
-                        if (ok && round == 0) {          // the first use of a K block waits for its copy
-                            ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
-                            k_par ^= 1u << kb;
-                        }
-                        if (!ok) break;
+                        const uint32_t sb = s_buf, cyc = s_cyc;
+                        const bool mine = (g & 1u) == me;
+                        ++g;
                         if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
+                        if (!mine) continue;
+                        if (cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (cyc - 1) & 1, abortp, a.status);
+                        // the K block's copy must have landed: in the second round too, where the
+                        // block may fall to the issuer that did not wait for it in the first
+                        if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
+                        if (!ok) break;
                         tcgen05_fence_after();
                         // K block kb sits (kb < 2 ? kb : kb + 2) tiles above the first prefetch slot;
                         // two k-steps of 32 over d = 64
@@ -327,7 +334,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     }
                 }
                 if (!ok) break;
-                tcgen05_commit(smem_u32(&bars.k_done));
+                k_par ^= (1u << kblocks) - 1u;               // every k_full[kb < kblocks] completed one phase
+                tcgen05_commit(smem_u32(&bars.k_done));      // both issuers: the barrier counts two
             }
         }
     } else if (warp == kPvWarp) {
