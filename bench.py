@@ -184,7 +184,7 @@ def run_fused(args):
 
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    wl = workloads.make_config(5)
+    wl = workloads.make_attention(12345, [int(v) for v in args.shape.split(",")]) if args.shape else workloads.make_config(5)
     Bt, H, L, d = wl.shape
     ctx = pkg.Context(0)
     ctx.hccs_params_upload(wl.theta, wl.n_design)
@@ -433,7 +433,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--shape", default="", help="B,H,Lq,Lk: time hccs_forward on seeded Gaussian rows of this "
-                                                "shape instead of a named workload")
+                                                "shape instead of a named workload (with --config 5: B,H,L,d "
+                                                "operands of the fused call)")
     ap.add_argument("--mode", default="u8div", choices=["u8div", "u8clb", "u16div", "u16clb"],
                     help="output type and reciprocal of hccs_forward (the headline is u8div)")
     ap.add_argument("--kernel-only", action="store_true",

@@ -373,7 +373,7 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
         memcpy(&e[4], &scale, sizeof(float));
         if (requant_shift <= 24) {
             const int sh = requant_shift, k = 24 - sh;
-            const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= 64*128*128 = 2^20
+            const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= d*128*128 <= 2^21
             int64_t lo = -lim, hi = lim;
             if (M > 0) {
                 lo = -((((int64_t)128 << sh) + R) / M);          // smallest accumulator that gives -128

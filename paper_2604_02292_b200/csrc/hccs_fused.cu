@@ -44,9 +44,10 @@ namespace {
 constexpr int kRowThreads = 512;           // four per query row
 constexpr int kThreads = 640;            // 16 row warps and four single-lane role warps
 constexpr int kTmaWarp = 16, kQkWarp = 17, kPvWarp = 18, kQk2Warp = 19;
-constexpr int kD = 64;                    // head dimension (bytes per Q/K/V row)
+constexpr int kHalf = 64;                 // operand rows are staged 64 bytes at a time (64-byte swizzle): d = 64 is one
+                                          // such half tile per Q, K or V tile, d = 128 two
 constexpr int kTile = 128;                // queries per CTA, keys per block
-constexpr int kTileBytes = kTile * kD;    // 8 KB: one Q, K or V tile
+constexpr int kHalfBytes = kTile * kHalf;  // 8 KB: 128 rows x 64 bytes
 constexpr int kPanelBlockBytes = kTile * 128;   // 16 KB: 128 rows x 128 keys of the panel
 constexpr int kMaxBlocks = 8;             // L <= 1024
 constexpr uint32_t kTmemCols = 512;       // S0 [0,128)  S1 [128,256)  S2 [256,384)  O [384,448)
@@ -195,11 +196,13 @@ struct FusedSmemBarriers {
     uint64_t o_full;
 };
 
-template <bool CLB, bool CAUSAL>
+template <int D, bool CLB, bool CAUSAL>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                        FusedArgs a, int num_tiles) {
+    constexpr int kHalves = D / kHalf;                    // half tiles per Q, K or V tile
+    constexpr int kTileBytes = kTile * D;                 // one Q, K or V tile: 8 or 16 KB
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) FusedSmemBarriers bars;
     __shared__ uint32_t tmem_base_slot;
@@ -257,14 +260,18 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             bool ok = true;
             // Q and the first two K blocks of a tile go to buffers of their own, so they can be
             // fetched while the previous tile is still in its softmax passes.
+            // one Q, K or V tile: its 64-byte column halves land one after the other
+            auto load_tile = [&](uint32_t dst, const CUtensorMap *map, int row, uint32_t bar) {
+                mbar_expect_tx(bar, kTileBytes);
+#pragma unroll
+                for (int h = 0; h < kHalves; ++h) tma_load_2d(dst + h * kHalfBytes, map, h * kHalf, row, bar);
+            };
             auto prefetch = [&](int tile) {
                 const int bh = tile / nblk, qt = tile % nblk;
                 const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
-                mbar_expect_tx(smem_u32(&bars.q_full), kTileBytes);
-                tma_load_2d(s_q, &map_q, 0, bh * a.L + qt * kTile, smem_u32(&bars.q_full));
+                load_tile(s_q, &map_q, bh * a.L + qt * kTile, smem_u32(&bars.q_full));
                 for (int kb = 0; kb < min(2, kblocks); ++kb) {
-                    mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
-                    tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
+                    load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
             };
             if ((int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
@@ -275,16 +282,14 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 if (it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (it - 1) & 1, abortp, a.status);
                 if (!ok) break;
                 for (int kb = 2; kb < kblocks; ++kb) {
-                    mbar_expect_tx(smem_u32(&bars.k_full[kb]), kTileBytes);
-                    tma_load_2d(k_slot(kb), &map_k, 0, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
+                    load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
                 // V takes the K buffer once the first contraction has read the last K block; Q and
                 // the first K blocks of the next tile are fetched as well
                 ok = mbar_wait(smem_u32(&bars.k_done), it & 1, abortp, a.status);
                 if (!ok) break;
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    mbar_expect_tx(smem_u32(&bars.v_full[kb]), kTileBytes);
-                    tma_load_2d(s_kv + kb * kTileBytes, &map_v, 0, bh * a.L + kb * kTile, smem_u32(&bars.v_full[kb]));
+                    load_tile(s_kv + kb * kTileBytes, &map_v, bh * a.L + kb * kTile, smem_u32(&bars.v_full[kb]));
                 }
                 if (tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
             }
@@ -326,10 +331,16 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         if (!ok) break;
                         tcgen05_fence_after();
                         // K block kb sits (kb < 2 ? kb : kb + 2) tiles above the first prefetch slot;
-                        // two k-steps of 32 over d = 64
+                        // two k-steps of 32 per 64-byte half of d
                         const uint32_t koff = (uint32_t)((kb < 2 ? kb : kb + 2) * kTileBytes) >> 4;
-                        tcgen05_mma_i8(tmem + sb * 128, make_u64(dq_lo, dq_hi), make_u64(dk_lo + koff, dk_hi), kIdescQK, 0);
-                        tcgen05_mma_i8(tmem + sb * 128, make_u64(dq_lo + 2, dq_hi), make_u64(dk_lo + koff + 2, dk_hi), kIdescQK, 1);
+#pragma unroll
+                        for (int h = 0; h < kHalves; ++h)
+#pragma unroll
+                            for (int ks = 0; ks < 2; ++ks) {
+                                const uint32_t off = (uint32_t)(h * kHalfBytes + ks * 32) >> 4;
+                                tcgen05_mma_i8(tmem + sb * 128, make_u64(dq_lo + off, dq_hi), make_u64(dk_lo + koff + off, dk_hi),
+                                               kIdescQK, (h | ks) != 0);
+                            }
                         tcgen05_commit(smem_u32(&bars.s_full[sb]));
                     }
                 }
@@ -362,9 +373,12 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint32_t poff = (uint32_t)(kb * kPanelBlockBytes + ks * 32) >> 4;
-                        const uint32_t voff = (uint32_t)((kb * kTile + ks * 32) * kD) >> 4;
-                        tcgen05_mma_i8(tmem + kTmemO, make_u64(dp_lo + poff, dp_hi), make_u64(dv_lo + voff, dv_hi), kIdescPV,
-                                       (kb | ks) != 0);
+#pragma unroll
+                        for (int h = 0; h < kHalves; ++h) {      // 64 output columns per half tile of V
+                            const uint32_t voff = (uint32_t)(kb * kTileBytes + h * kHalfBytes + ks * 32 * kHalf) >> 4;
+                            tcgen05_mma_i8(tmem + kTmemO + h * kHalf, make_u64(dp_lo + poff, dp_hi), make_u64(dv_lo + voff, dv_hi),
+                                           kIdescPV, (kb | ks) != 0);
+                        }
                     }
                 }
                 if (!ok) break;
@@ -619,16 +633,20 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if (ok) ok = mbar_wait(smem_u32(&bars.o_full), it & 1, abortp, a.status);
             if (ok) {
                 tcgen05_fence_after();
-                uint32_t acc[16];
-                tmem_ld16(tmem + lane_addr + kTmemO + grp * 16, acc);
+                constexpr int kCols = D / 4;                      // columns of O per thread: 16 or 32
+                uint32_t acc[kCols];
+                if constexpr (kCols == 16) tmem_ld16(tmem + lane_addr + kTmemO + grp * kCols, acc);
+                else tmem_ld32(tmem + lane_addr + kTmemO + grp * kCols, acc);
                 if (a.out_f32) {                                  // optional dequantised view of O
 #pragma unroll
-                    for (int g = 0; g < 16; ++g) acc[g] = __float_as_uint(__int2float_rn((int)acc[g]) * out_scale);
+                    for (int g = 0; g < kCols; ++g) acc[g] = __float_as_uint(__int2float_rn((int)acc[g]) * out_scale);
                 }
-                uint8_t *o_stage = panel + (grp >> 1) * kOBoxBytes + t * 128;
+                // column c of the tile sits in box c / 32, 16-byte chunk (c % 32) / 4 of its row
+                const int c0 = grp * kCols;
+                uint8_t *o_stage = panel + (c0 >> 5) * kOBoxBytes + t * 128;
 #pragma unroll
-                for (int g = 0; g < 4; ++g)
-                    *reinterpret_cast<uint4 *>(o_stage + ((((grp & 1) * 4 + g) ^ swz) << 4)) =
+                for (int g = 0; g < kCols / 4; ++g)
+                    *reinterpret_cast<uint4 *>(o_stage + (((((c0 & 31) >> 2) + g) ^ swz) << 4)) =
                         make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
                 tcgen05_fence_before();
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -636,8 +654,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if (tid == 0) leave_flag = *abortp;                   // one reader, so that all row threads agree
             asm volatile("bar.sync 1, 512;" ::: "memory");
             if (tid == 0 && !*(volatile int *)&leave_flag) {
-                tma_store_3d(&map_o, 0, q0, bh, s_p);
-                tma_store_3d(&map_o, 32, q0, bh, s_p + kOBoxBytes);
+#pragma unroll
+                for (int b = 0; b < D / 32; ++b) tma_store_3d(&map_o, 32 * b, q0, bh, s_p + b * kOBoxBytes);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
             // leave the loop together (the flag was sampled once, before the barrier above)
@@ -675,26 +693,26 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// [rows, 64] uint8 tensor, boxes of 128 rows x 64 bytes, 64-byte swizzle.
-bool make_tile_map(CUtensorMap *map, const void *ptr, uint64_t rows) {
+// [rows, d] uint8 tensor, boxes of 128 rows x 64 bytes (one column half of a tile), 64-byte swizzle.
+bool make_tile_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint32_t d) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)kD};
-    const cuuint32_t box[2] = {(cuuint32_t)kD, (cuuint32_t)kTile};
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)d};
+    const cuuint32_t box[2] = {(cuuint32_t)kHalf, (cuuint32_t)kTile};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// O as [B*H][L][64] 32-bit words, boxes of 128 rows x 32 words, 128-byte swizzle.  Three dimensions, so
+// O as [B*H][L][d] 32-bit words, boxes of 128 rows x 32 words, 128-byte swizzle.  Three dimensions, so
 // that a tile of the last, partial row block of a head stops at the head's end.
-bool make_output_map(CUtensorMap *map, const void *ptr, uint64_t heads, uint64_t L) {
+bool make_output_map(CUtensorMap *map, const void *ptr, uint64_t heads, uint64_t L, uint32_t d) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)L, (cuuint64_t)heads};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 4, (cuuint64_t)kD * 4 * L};
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)L, (cuuint64_t)heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)d * 4, (cuuint64_t)d * 4 * L};
     const cuuint32_t box[3] = {32, (cuuint32_t)kTile, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(ptr), dims, strides, box, estr,
@@ -702,14 +720,15 @@ bool make_output_map(CUtensorMap *map, const void *ptr, uint64_t heads, uint64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool CLB, bool CAUSAL>
+template <int D, bool CLB, bool CAUSAL>
 cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mo,
                            const FusedArgs &a, cudaStream_t st) {
     const int nblk = (a.L + kTile - 1) / kTile;
+    constexpr size_t kTileBytes = (size_t)kTile * D;
     size_t panel = (size_t)kTile * nblk * kTile;
-    if (panel < 2 * (size_t)kOBoxBytes) panel = 2 * (size_t)kOBoxBytes;   // the staged O boxes reuse the panel
-    const size_t smem = 1024 + 3 * (size_t)kTileBytes + (size_t)nblk * kTileBytes + panel;
-    auto kernel = fused_attention_kernel<CLB, CAUSAL>;
+    if (panel < (D / 32) * (size_t)kOBoxBytes) panel = (D / 32) * (size_t)kOBoxBytes;   // the staged O boxes reuse the panel
+    const size_t smem = 1024 + 3 * kTileBytes + (size_t)nblk * kTileBytes + panel;
+    auto kernel = fused_attention_kernel<D, CLB, CAUSAL>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t tiles = (int64_t)a.B * a.H * nblk;
@@ -723,23 +742,32 @@ cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const C
 
 }  // namespace
 
+// d = 64 with up to 1024 keys, d = 128 with up to 512 (K, V and the panel share the SM's shared memory).
 bool fused_shape_supported(int32_t L, int32_t d) {
-    return d == kD && L >= 1 && L <= kTile * kMaxBlocks;
+    return L >= 1 && ((d == 64 && L <= kTile * kMaxBlocks) || (d == 128 && L <= kTile * kMaxBlocks / 2));
 }
 
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches) {
     CUtensorMap mq, mk, mv, mo;
     const uint64_t rows = (uint64_t)a.B * a.H * a.L;
-    if (!make_tile_map(&mq, a.Q, rows) || !make_tile_map(&mk, a.K, rows) || !make_tile_map(&mv, a.V, rows) ||
-        !make_output_map(&mo, a.O, (uint64_t)a.B * a.H, (uint64_t)a.L))
+    if (!fused_shape_supported(a.L, a.d)) return cudaErrorInvalidValue;
+    if (!make_tile_map(&mq, a.Q, rows, a.d) || !make_tile_map(&mk, a.K, rows, a.d) || !make_tile_map(&mv, a.V, rows, a.d) ||
+        !make_output_map(&mo, a.O, (uint64_t)a.B * a.H, (uint64_t)a.L, a.d))
         return cudaErrorInvalidValue;
     cudaError_t e;
     // the masked instantiation also serves L that is no multiple of 128 (padding keys in the last block)
     const bool clb = (a.flags & HCCS_RECIP_CLB) != 0, causal = (a.flags & HCCS_CAUSAL) != 0 || a.L % kTile != 0;
-    if (!clb && !causal) e = launch_variant<false, false>(mq, mk, mv, mo, a, stream);
-    else if (clb && !causal) e = launch_variant<true, false>(mq, mk, mv, mo, a, stream);
-    else if (!clb && causal) e = launch_variant<false, true>(mq, mk, mv, mo, a, stream);
-    else e = launch_variant<true, true>(mq, mk, mv, mo, a, stream);
+    if (a.d == 64) {
+        if (!clb && !causal) e = launch_variant<64, false, false>(mq, mk, mv, mo, a, stream);
+        else if (clb && !causal) e = launch_variant<64, true, false>(mq, mk, mv, mo, a, stream);
+        else if (!clb && causal) e = launch_variant<64, false, true>(mq, mk, mv, mo, a, stream);
+        else e = launch_variant<64, true, true>(mq, mk, mv, mo, a, stream);
+    } else {
+        if (!clb && !causal) e = launch_variant<128, false, false>(mq, mk, mv, mo, a, stream);
+        else if (clb && !causal) e = launch_variant<128, true, false>(mq, mk, mv, mo, a, stream);
+        else if (!clb && causal) e = launch_variant<128, false, true>(mq, mk, mv, mo, a, stream);
+        else e = launch_variant<128, true, true>(mq, mk, mv, mo, a, stream);
+    }
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }

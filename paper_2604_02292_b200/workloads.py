@@ -164,6 +164,19 @@ def make_config(c: int, batch: int | None = None) -> Workload:
     raise ValueError("config index must be 1..5")
 
 
+def make_attention(seed: int, shape) -> Workload:
+    """Fused-attention operands of any [B, H, L, d], drawn like workload 5's: uniform int8 in
+    [-64, 63], theta in the band for L keys, multipliers scaled by 64 / d so that the logits keep
+    workload 5's spread."""
+    Bt, H, L, d = (int(v) for v in shape)
+    rng = np.random.Generator(np.random.PCG64(int(seed)))
+    theta = sample_theta(rng, H, L)
+    mult = (rng.integers(768, 3841, size=H) * 64 // d).astype(np.int32)
+    Q, K, V = (rng.integers(-64, 64, size=(Bt, H, L, d), dtype=np.int8) for _ in range(3))
+    return Workload("attention" + "x".join(str(v) for v in (Bt, H, L, d)), (Bt, H, L, d), 0, L, theta,
+                    Q=Q, K=K, V=V, requant_mult=mult, requant_shift=20)
+
+
 def make_rows(seed: int, shape, n_design: int | None = None, kind: str = "gauss",
               flags: int = 0) -> Workload:
     """Small seeded standalone workload of any shape, for parity and edge-case tests.

@@ -39,6 +39,34 @@ def test_small_heads(hccs, oracle, L, flags):
     assert_same(got, want, f"fused L={L} flags={flags}")
 
 
+@pytest.mark.parametrize("L", [1, 100, 128, 384, 500, 512])
+@pytest.mark.parametrize("flags", [0, 4, 6])
+def test_head_dimension_128(hccs, oracle, L, flags):
+    """d = 128 (two 64-byte column halves per Q, K and V tile, 128 output columns), up to 512 keys,
+    full-range int8 operands: |acc| reaches 2^21."""
+    rng = np.random.default_rng(4000 + L + flags)
+    Bt, H, d = 2, 2, 128
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
+    theta = hccs.workloads.sample_theta(rng, H, 512)
+    mult = rng.integers(400, 1500, size=H).astype(np.int32)
+    got = _run(hccs, Q, K, V, theta, mult, 20, 512, flags)
+    want = oracle.attention(Q, K, V, mult, 20, theta, oracle_mode(oracle, flags), threads=8)
+    assert_same(got, want, f"fused d=128 L={L} flags={flags}")
+
+
+def test_head_dimension_128_many_tiles_and_wide_shift(hccs, oracle):
+    """More tiles than SMs (persistent CTAs take several), and the 64-bit requantisation flow."""
+    rng = np.random.default_rng(4100)
+    Bt, H, L, d = 10, 5, 512, 128
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d))
+    theta = hccs.workloads.sample_theta(rng, H, L)
+    for sh, lo, hi in ((21, 768, 3841), (28, 4096, 8192)):
+        mult = rng.integers(lo, hi, size=H).astype(np.int32)
+        got = _run(hccs, Q, K, V, theta, mult, sh, L)
+        want = oracle.attention(Q, K, V, mult, sh, theta, 0, threads=16)
+        assert_same(got, want, f"fused d=128 sh={sh}")
+
+
 def test_full_range_int8_and_saturating_requant(hccs, oracle):
     """Operands over all of int8 (|acc| up to 2^20) with multipliers that drive the logits into
     the int8 clamp; also OUT_SHIFT = 1 and a table designed for more keys than the call uses."""
@@ -90,7 +118,7 @@ def test_unsupported_shapes_are_refused(hccs):
     import torch
     ctx = hccs.Context(0)
     ctx.hccs_params_upload([(31, 1, 20)] * 2, 1024)
-    for L, d in ((128, 32), (2048, 64), (1040, 64)):
+    for L, d in ((128, 32), (2048, 64), (1040, 64), (640, 128), (128, 96)):
         q = torch.zeros((1, 2, L, d), dtype=torch.int8, device="cuda")
         o = torch.zeros((1, 2, L, d), dtype=torch.int32, device="cuda")
         with pytest.raises(hccs.HccsError) as ei:
@@ -104,14 +132,15 @@ def test_unsupported_shapes_are_refused(hccs):
     ctx.close()
 
 
-def test_fp32_dequantised_output(hccs, oracle):
+@pytest.mark.parametrize("d", [64, 128])
+def test_fp32_dequantised_output(hccs, oracle, d):
     """O_f32 = float(int32 O) * scale_h: within 1e-6 relative of the exact product (fp64 from the oracle)."""
     import torch
     rng = np.random.default_rng(9)
-    Bt, H, L, d = 1, 3, 384, 64
+    Bt, H, L = 1, 3, 384
     Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
     theta = hccs.workloads.sample_theta(rng, H, L)
-    mult = rng.integers(768, 3841, size=H).astype(np.int32)
+    mult = rng.integers(768, 3841, size=H).astype(np.int32) // (d // 64)
     scale = np.array([0.03125 / 255, 1.7e-3, 0.4], dtype=np.float32)
     ctx = hccs.Context(0)
     ctx.hccs_params_upload(theta, L)
