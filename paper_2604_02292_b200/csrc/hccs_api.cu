@@ -363,7 +363,7 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     HCCS_CUDA(ctx, cudaEventSynchronize(ctx->mult_copied));
     // Per head: {multiplier, and for shifts up to 24 the constants of the single-multiply
     // requantisation: multiplier << k, offset, -lo, hi - lo} (see hccs_fused.cu, phase 1), then the
-    // fp32 output scale; eight 32-bit words per head.
+    // fp32 output scale, a spare word and 1 / multiplier as a double; eight 32-bit words per head.
     for (int32_t h = 0; h < H; ++h) {
         const int64_t M = requant_mult[h];
         int32_t *e = ctx->h_mult + 8 * h;
@@ -371,6 +371,8 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
         e[1] = e[2] = e[3] = e[5] = e[6] = e[7] = 0;
         const float scale = out_scale ? out_scale[h] : 1.0f;
         memcpy(&e[4], &scale, sizeof(float));
+        const double inv_m = M > 0 ? 1.0 / (double)M : 0.0;      // words 6 and 7
+        memcpy(&e[6], &inv_m, sizeof(double));
         if (requant_shift <= 24) {
             const int sh = requant_shift, k = 24 - sh;
             const int64_t R = (int64_t)1 << (sh - 1), lim = (int64_t)1 << 21;   // |acc| <= d*128*128 <= 2^21

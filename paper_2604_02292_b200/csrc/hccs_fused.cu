@@ -403,6 +403,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const HeadEntry th = a.table[head];
             const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head);   // host-prepared constants
             const float out_scale = __int_as_float(a.requant_mult[8 * head + 4]);
+            const double inv_m = *reinterpret_cast<const double *>(a.requant_mult + 8 * head + 6);   // 1 / M_h
             // valid keys of this row: all L of them, or the causal prefix (keys at and beyond L exist
             // only as padding of the last block when L is no multiple of 128)
             const int nv = (CAUSAL && causal) ? min(q0 + t + 1, a.L) : a.L;
@@ -466,27 +467,18 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 xmax = max(max(part_max[0][t], part_max[1][t]), max(part_max[2][t], part_max[3][t]));
                 cm = th.D - xmax;
 
-                // lo_t = clamp(ceil((t*2^sh - R) / M), lo, hi): two single-precision estimates of the
-                // quotient (the second on the remainder of the first, which leaves at most one unit
-                // of error) and integer corrections
+                // lo_t = clamp(ceil((t*2^sh - R) / M), lo, hi).  |t*2^sh - R| < 2^33 and M < 2^13: the product
+                // with the host's double 1/M is within 2^-18 of the quotient, whose fraction is 0 or at
+                // least 1/M, so rounding to nearest gives the ceiling or one less
                 const int sh = a.requant_shift, kk = 24 - sh;
                 const int M = (int)(mk >> kk), lo = -neg_lo, hi = lo + span;
                 const int64_t R = (int64_t)1 << (sh - 1);
-                const int64_t want = (int64_t)(-cm) * ((int64_t)1 << sh);       // t * 2^sh
+                const int64_t num = (int64_t)(-cm) * ((int64_t)1 << sh) - R;    // t * 2^sh - R
                 int lo_t = lo;
                 if (M > 0) {
-                    const float inv_m = 1.0f / (float)M;
-                    const int64_t num = want - R;
-                    int q = (int)fminf(fmaxf(floorf((float)num * inv_m), (float)(lo - 1)), (float)(hi + 1));
-                    q += (int)fminf(fmaxf(floorf((float)(num - (int64_t)q * M) * inv_m), -8388608.0f), 8388608.0f);
-                    q = min(max(q, lo - 4), hi + 4);
-#pragma unroll
-                    for (int c = 0; c < 2; ++c)
-                        if ((int64_t)q * M < num) ++q;
-#pragma unroll
-                    for (int c = 0; c < 2; ++c)
-                        if ((int64_t)(q - 1) * M >= num) --q;
-                    lo_t = min(max(q, lo), hi);
+                    int64_t q = __double2ll_rn(__ll2double_rn(num) * inv_m);
+                    if (q * M < num) ++q;
+                    lo_t = (int)min(max(q, (int64_t)lo), (int64_t)hi);
                 }
                 const int neg_lo_t = -lo_t, span_t = hi - lo_t;
                 const uint32_t ck_t =
