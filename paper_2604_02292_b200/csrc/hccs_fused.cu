@@ -288,10 +288,13 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 // the first K blocks of the next tile are fetched as well
                 ok = mbar_wait(smem_u32(&bars.k_done), it & 1, abortp, a.status);
                 if (!ok) break;
+                // (a thread gets through one copy per ~600 cycles: the next tile's Q and K go after the
+                // first V blocks, early enough for its first round to start behind the probability pass)
                 for (int kb = 0; kb < kblocks; ++kb) {
+                    if (kb == 2 && tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
                     load_tile(s_kv + kb * kTileBytes, &map_v, bh * a.L + kb * kTile, smem_u32(&bars.v_full[kb]));
                 }
-                if (tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
+                if (kblocks <= 2 && tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
             }
         }
     } else if (warp == kQkWarp || warp == kQk2Warp) {
@@ -394,6 +397,27 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         const int swz = t & 7;
         uint32_t s_buf = 0, s_cyc = 0;                       // S buffer of the next block and its use count
         bool ok = true;
+        // one S block of the first round: the running maximum of the row's raw accumulators
+        auto first_round_block = [&](int kb, int nv_row, int &amax) {
+            const uint32_t sb = s_buf;
+            ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
+            if (!ok) return;
+            if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
+            tcgen05_fence_after();
+            uint32_t acc[32];
+            tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+            const int c0 = kb * kTile + grp * 32;
+            if (CAUSAL && c0 + 32 > nv_row) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    if (c0 + e >= nv_row) acc[e] = (uint32_t)(-(1 << 30));
+            }
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) amax = __vimax3_s32(amax, (int)acc[e], (int)acc[e + 1]);
+            tcgen05_fence_before();
+            mbar_arrive(smem_u32(&bars.s_free[sb]));
+        };
+        int amax_carry = -(1 << 30), r1_carry = 0;           // first-round blocks of a tile taken ahead of it
 
         for (int tile = blockIdx.x, it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
             const int bh = tile / nblk, qt = tile % nblk;
@@ -440,26 +464,9 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if (two_rounds) {
                 const uint32_t mk = (uint32_t)rq.x, ck = (uint32_t)rq.y;
                 const int neg_lo = rq.z, span = rq.w;
-                int amax = -(1 << 30);
-                for (int kb = 0; ok && kb < kblocks; ++kb) {
-                    const uint32_t sb = s_buf;
-                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
-                    if (!ok) break;
-                    if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
-                    tcgen05_fence_after();
-                    uint32_t acc[32];
-                    tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
-                    const int c0 = kb * kTile + grp * 32;
-                    if (CAUSAL && c0 + 32 > nv) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c0 + e >= nv) acc[e] = (uint32_t)(-(1 << 30));
-                    }
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) amax = __vimax3_s32(amax, (int)acc[e], (int)acc[e + 1]);
-                    tcgen05_fence_before();
-                    mbar_arrive(smem_u32(&bars.s_free[sb]));
-                }
+                // (the first two blocks were taken at the end of the previous tile, see below)
+                int amax = amax_carry;
+                for (int kb = r1_carry; ok && kb < kblocks; ++kb) first_round_block(kb, nv, amax);
                 xmax = (int)((uint32_t)__viaddmin_s32_relu(amax, neg_lo, span) * mk + ck) >> 24;
                 part_max[grp][t] = xmax;
                 if (tid == 0 && it > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -613,6 +620,18 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 // the tensor core reads the panel through the async proxy: hand this block over
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive(smem_u32(&bars.p_ready[kb]));
+            }
+
+            // ---- while the last P.V block finishes: the first round of the NEXT tile over its first two
+            // key blocks, whose K tiles (and Q) were prefetched and whose S blocks the tensor core has
+            // produced meanwhile (the other K tiles can only be fetched once V is no longer needed)
+            amax_carry = -(1 << 30);
+            r1_carry = 0;
+            if (two_rounds && tile + (int)gridDim.x < num_tiles) {
+                const int qt_n = (tile + (int)gridDim.x) % nblk;
+                const int kblocks_n = (CAUSAL && causal) ? qt_n + 1 : nblk;
+                const int nv_n = (CAUSAL && causal) ? min(qt_n * kTile + t + 1, a.L) : a.L;
+                for (; ok && r1_carry < min(2, kblocks_n); ++r1_carry) first_round_block(r1_carry, nv_n, amax_carry);
             }
 
             // ---- phase 4: O out of tensor memory.  A thread holds 16 columns of its row; writing them
