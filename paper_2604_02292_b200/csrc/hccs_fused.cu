@@ -17,13 +17,13 @@
 //   * V is used as stored ([key][64], keys outermost): that is exactly the MN-major, 64-byte
 //     swizzled B operand, so no transposition is needed.
 //
-// Warp roles (640 threads): warps 0-15 are row warps, four threads per query row (threads t,
+// Warp roles (672 threads): warps 0-15 are row warps, four threads per query row (threads t,
 // t + 128, t + 256, t + 384 own row t mod 128; TMEM lane quarter = warp index mod 4): bits 7-8
 // of the thread index select which 32 of the 128 keys of every block the thread handles, so all
 // row threads work on the same block while the tensor core fills the other S buffers.
 // The four exchange their partial row max and row sum through shared memory; the many warps are
-// what hides the latency of the dependent integer chains.  Four more warps each run one
-// single-lane role on a scheduler of their own: warp 16 issues every TMA load, warps 17 and 19
+// what hides the latency of the dependent integer chains.  Five more warps each run one
+// single-lane role: warps 16 and 20 issue the TMA loads (alternate blocks), warps 17 and 19
 // the first contraction (alternate blocks), warp 18 the second (one thread doing it all fell
 // behind the row warps: its serial chain of waits, descriptor arithmetic and issues cost several
 // hundred cycles per block).
@@ -42,8 +42,8 @@ namespace hccs {
 namespace {
 
 constexpr int kRowThreads = 512;           // four per query row
-constexpr int kThreads = 640;            // 16 row warps and four single-lane role warps
-constexpr int kTmaWarp = 16, kQkWarp = 17, kPvWarp = 18, kQk2Warp = 19;
+constexpr int kThreads = 672;            // 16 row warps and five single-lane role warps
+constexpr int kTmaWarp = 16, kQkWarp = 17, kPvWarp = 18, kQk2Warp = 19, kTma2Warp = 20;
 constexpr int kHalf = 64;                 // operand rows are staged 64 bytes at a time (64-byte swizzle): d = 64 is one
                                           // such half tile per Q, K or V tile, d = 128 two
 constexpr int kTile = 128;                // queries per CTA, keys per block
@@ -254,9 +254,12 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     // A CTA walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every mbarrier completes
     // one phase per use, so both sides count their uses (per barrier, because a causal tile uses
     // only its first qt + 1 key blocks) and wait on the parity of that count.
-    if (warp == kTmaWarp) {
-        // ===================================================== copy thread: every TMA load
+    if (warp == kTmaWarp || warp == kTma2Warp) {
+        // ===================================================== copy threads: every TMA load.  A thread gets
+        // through one copy per ~600 cycles whatever its size, copies of different warps overlap: the
+        // first thread takes Q and the even K and V blocks, the second the odd ones.
         if (lane == 0) {
+            const int me = warp == kTmaWarp ? 0 : 1;
             bool ok = true;
             // Q and the first two K blocks of a tile go to buffers of their own, so they can be
             // fetched while the previous tile is still in its softmax passes.
@@ -274,27 +277,26 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
             };
-            if ((int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
+            if (me == 0 && (int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int bh = tile / nblk, qt = tile % nblk;
                 const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
                 // the other K blocks land where the previous tile's V sits: wait for its last MMA
                 if (it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (it - 1) & 1, abortp, a.status);
                 if (!ok) break;
-                for (int kb = 2; kb < kblocks; ++kb) {
+                for (int kb = 2 + me; kb < kblocks; kb += 2) {
                     load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
                 // V takes the K buffer once the first contraction has read the last K block; Q and
                 // the first K blocks of the next tile are fetched as well
                 ok = mbar_wait(smem_u32(&bars.k_done), it & 1, abortp, a.status);
                 if (!ok) break;
-                // (a thread gets through one copy per ~600 cycles: the next tile's Q and K go after the
-                // first V blocks, early enough for its first round to start behind the probability pass)
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (kb == 2 && tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
+                // (the next tile's Q and K go after the first V block, early enough for its first round
+                // to start behind the probability pass)
+                for (int kb = me; kb < kblocks; kb += 2) {
                     load_tile(s_kv + kb * kTileBytes, &map_v, bh * a.L + kb * kTile, smem_u32(&bars.v_full[kb]));
+                    if (kb == 0 && tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
                 }
-                if (kblocks <= 2 && tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
             }
         }
     } else if (warp == kQkWarp || warp == kQk2Warp) {
