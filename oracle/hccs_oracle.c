@@ -210,6 +210,9 @@ int64_t hccs_oracle_requant(int64_t acc, int64_t M, int64_t sh)
  * int32 [Bt,H,L,d].  x_tmp, p_tmp: L entries each; valid_tmp: L bytes.
  * logits_out / probs_out (may be NULL) receive the intermediate int8 logits and
  * uint8 probabilities of the computed rows, laid out [Bt,H,L,L].
+ * key_len (may be NULL): int32 [Bt]; keys at and beyond key_len[b] are padding of
+ * batch entry b: like causally masked keys they take no part in max and sum and get
+ * probability 0 (masking is not in the paper; the valid keys are always a prefix).
  */
 int hccs_oracle_attention(const int8_t *Q, const int8_t *K, const int8_t *V, int32_t *O,
                           const int32_t *M, int64_t sh, const int32_t *params,
@@ -217,7 +220,7 @@ int hccs_oracle_attention(const int8_t *Q, const int8_t *K, const int8_t *V, int
                           int mode, int64_t out_shift,
                           int64_t bh_begin, int64_t bh_end, int64_t q_begin, int64_t q_end,
                           int8_t *x_tmp, int64_t *p_tmp, uint8_t *valid_tmp,
-                          int8_t *logits_out, uint8_t *probs_out)
+                          int8_t *logits_out, uint8_t *probs_out, const int32_t *key_len)
 {
     int64_t bh, i, j, c;
     (void)Bt;
@@ -235,8 +238,16 @@ int hccs_oracle_attention(const int8_t *Q, const int8_t *K, const int8_t *V, int
                 for (c = 0; c < d; ++c) acc += (int64_t)q[i * d + c] * (int64_t)k[j * d + c];
                 x_tmp[j] = (int8_t)hccs_oracle_requant(acc, M[h], sh);
             }
-            if (mode & ORACLE_MODE_CAUSAL) {
-                for (j = 0; j < L; ++j) valid_tmp[j] = (uint8_t)(j <= i);
+            if ((mode & ORACLE_MODE_CAUSAL) || key_len) {
+                /* valid keys form a prefix: the causal rule and / or the batch entry's key length */
+                int64_t limit = L;
+                if (key_len) {
+                    limit = key_len[bh / H];
+                    if (limit < 0) limit = 0;
+                    if (limit > L) limit = L;
+                }
+                for (j = 0; j < L; ++j)
+                    valid_tmp[j] = (uint8_t)(j < limit && (!(mode & ORACLE_MODE_CAUSAL) || j <= i));
                 valid = valid_tmp;
             }
             hccs_oracle_row(x_tmp, valid, L, params[3 * h + 0], params[3 * h + 1],

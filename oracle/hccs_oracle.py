@@ -64,7 +64,7 @@ def lib() -> ctypes.CDLL:
             L.hccs_oracle_requant.restype = _i64
             L.hccs_oracle_attention.argtypes = [_p, _p, _p, _p, _p, _i64, _p,
                                                 _i64, _i64, _i64, _i64, ctypes.c_int, _i64,
-                                                _i64, _i64, _i64, _i64, _p, _p, _p, _p, _p]
+                                                _i64, _i64, _i64, _i64, _p, _p, _p, _p, _p, _p]
             L.hccs_oracle_attention.restype = ctypes.c_int
             _lib = L
     return _lib
@@ -139,12 +139,13 @@ def forward(logits, params, mode: int = 0, out_shift: int = 0, threads: int = 1,
 
 
 def attention(Q, K, V, M, sh, params, mode: int = 0, out_shift: int = 0, threads: int = 1,
-              bh_range=None, q_range=None, want_intermediates: bool = False):
+              bh_range=None, q_range=None, want_intermediates: bool = False, key_len=None):
     """Integer attention Q.K^T -> requant -> HCCS (u8) -> P.V for int8 [B,H,L,d] inputs.
 
     Returns O int32 [B,H,L,d] (and, if asked, the int8 logits and uint8
     probabilities [B,H,L,L]).  Only slices in ``bh_range`` / rows in ``q_range``
-    are computed; the rest stay zero.
+    are computed; the rest stay zero.  ``key_len`` (int32 [B], optional): keys at
+    and beyond key_len[b] are padding of batch entry b and take no part.
     """
     Q = np.ascontiguousarray(Q, dtype=np.int8)
     K = np.ascontiguousarray(K, dtype=np.int8)
@@ -152,6 +153,7 @@ def attention(Q, K, V, M, sh, params, mode: int = 0, out_shift: int = 0, threads
     Bt, H, Lx, d = Q.shape
     pa = _params_array(params, H)
     Ma = np.ascontiguousarray(M, dtype=np.int32)
+    kl = None if key_len is None else np.ascontiguousarray(key_len, dtype=np.int32).reshape(Bt)
     O = np.zeros((Bt, H, Lx, d), dtype=np.int32)
     lg = np.zeros((Bt, H, Lx, Lx), dtype=np.int8) if want_intermediates else None
     pr = np.zeros((Bt, H, Lx, Lx), dtype=np.uint8) if want_intermediates else None
@@ -165,7 +167,7 @@ def attention(Q, K, V, M, sh, params, mode: int = 0, out_shift: int = 0, threads
         v_tmp = np.zeros(Lx, dtype=np.uint8)
         rc = L.hccs_oracle_attention(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(Ma), sh, _ptr(pa),
                                      Bt, H, Lx, d, mode, out_shift, a, b, q0, q1,
-                                     _ptr(x_tmp), _ptr(p_tmp), _ptr(v_tmp), _ptr(lg), _ptr(pr))
+                                     _ptr(x_tmp), _ptr(p_tmp), _ptr(v_tmp), _ptr(lg), _ptr(pr), _ptr(kl))
         if rc != 0:
             raise OverflowError(f"oracle attention failed rc={rc}")
 

@@ -57,3 +57,39 @@ def test_attention_matches_matrix_route():
     assert (O_part.reshape(-1, L, d)[2:5, 3:11] == O_all.reshape(-1, L, d)[2:5, 3:11]).all()
     assert not O_part.reshape(-1, L, d)[:2].any() and not O_part.reshape(-1, L, d)[2:5, :3].any()
     assert (orc.attention(Q, K, V, M, sh, theta, 0, threads=4) == O_all).all()
+
+
+def test_key_length_mask_equals_attention_over_the_truncated_keys():
+    """Padding keys take no part: attention with key_len[b] = n must equal attention over the first
+    n keys and values alone (for the queries both have), also under the causal rule; n = 0 gives
+    zeros and n >= L changes nothing."""
+    rng = np.random.default_rng(31)
+    Bt, H, L, d = 4, 2, 24, 8
+    Q, K, V = (rng.integers(-128, 128, size=(Bt, H, L, d), dtype=np.int8) for _ in range(3))
+    theta = np.array([[200, 3, 40], [120, 1, 90]], dtype=np.int32)
+    M = np.array([900, 3000], dtype=np.int32)
+    key_len = np.array([7, 0, 24, 31], dtype=np.int32)
+    for mode in (0, orc.MODE_CAUSAL, orc.MODE_CLB):
+        got = orc.attention(Q, K, V, M, 12, theta, mode, key_len=key_len)
+        full = orc.attention(Q, K, V, M, 12, theta, mode)
+        for b in range(Bt):
+            n = int(min(max(key_len[b], 0), L))
+            if n == 0:
+                assert (got[b] == 0).all()
+                continue
+            if n == L:
+                assert np.array_equal(got[b], full[b])
+                continue
+            # the same queries against the first n keys only: a call of its own on sliced tensors
+            Qb = np.ascontiguousarray(Q[b:b + 1, :, :n]); Kb = np.ascontiguousarray(K[b:b + 1, :, :n])
+            Vb = np.ascontiguousarray(V[b:b + 1, :, :n])
+            want = orc.attention(Qb, Kb, Vb, M, 12, theta, mode)
+            assert np.array_equal(got[b, :, :n], want[0]), (mode, b)
+            if not mode & orc.MODE_CAUSAL:
+                # queries beyond n still attend to the n keys: check one against a by-hand row
+                i = L - 1
+                for h in range(H):
+                    acc = Q[b, h, i].astype(np.int64) @ K[b, h, :n].astype(np.int64).T
+                    x = np.array([orc.requant(int(a_), int(M[h]), 12) for a_ in acc], dtype=np.int8)
+                    p = orc.forward(x.reshape(1, 1, 1, n), theta[h:h + 1], mode).reshape(n).astype(np.int64)
+                    assert np.array_equal(got[b, h, i], (p @ V[b, h, :n].astype(np.int64)).astype(np.int32))
