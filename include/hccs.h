@@ -163,6 +163,20 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
                                    uint32_t flags, void *cuda_stream);
 
 /*
+ * hccs_attention_fused with a key-padding mask: key_len is a DEVICE int32 [B] array; keys at and
+ * beyond key_len[b] (clamped to 0..L) of batch entry b are padding: like causally masked keys they
+ * take no part in the row maximum and the row sum and get probability 0, so O is the attention over
+ * the first key_len[b] keys alone; a batch entry with key length 0 gets O = 0.  Combines with
+ * HCCS_CAUSAL.  Everything else as hccs_attention_fused.  (Masking is not in the paper, whose
+ * encoder workloads are padded to a fixed length, Section "Models and tasks".)
+ */
+hccs_status_t hccs_attention_fused_keylen(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                          const int8_t *V, int32_t *O, const int32_t *key_len,
+                                          const int32_t *requant_mult, int32_t requant_shift,
+                                          int32_t B, int32_t H, int32_t L, int32_t d,
+                                          uint32_t flags, void *cuda_stream);
+
+/*
  * hccs_attention_fused with a dequantised fp32 output: O[b,h,i,:] = float(int32 accumulator) *
  * out_scale[h] (HOST float [H]; e.g. the V quantisation step divided by 255).  The integer result
  * is exact; the two fp32 roundings keep the relative error below 2^-23.  O is device float

@@ -337,7 +337,7 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
 
 // Shared by the int32 and the fp32 entry points: out_scale == NULL means int32 output.
 static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K, const int8_t *V, void *O,
-                                  const float *out_scale, const int32_t *requant_mult,
+                                  const float *out_scale, const int32_t *key_len, const int32_t *requant_mult,
                                   int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
                                   uint32_t flags, void *cuda_stream) {
     if (!ctx || B < 0 || H < 0 || L < 0 || d < 0) return HCCS_ERR_INVALID_ARG;
@@ -398,6 +398,7 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     a.requant_mult = ctx->d_mult;
     a.status = ctx->d_status;
     a.out_f32 = out_scale ? 1 : 0;
+    a.key_len = key_len;
     a.requant_shift = requant_shift;
     a.B = B; a.H = H; a.L = L; a.d = d;
     a.out_shift = ctx->out_shift;
@@ -410,7 +411,16 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
                                    const int8_t *V, int32_t *O, const int32_t *requant_mult,
                                    int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
                                    uint32_t flags, void *cuda_stream) {
-    return fused_common(ctx, Q, K, V, O, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+    return fused_common(ctx, Q, K, V, O, nullptr, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+}
+
+hccs_status_t hccs_attention_fused_keylen(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                          const int8_t *V, int32_t *O, const int32_t *key_len,
+                                          const int32_t *requant_mult, int32_t requant_shift,
+                                          int32_t B, int32_t H, int32_t L, int32_t d,
+                                          uint32_t flags, void *cuda_stream) {
+    if (!key_len && (int64_t)B * H * L * d != 0) return HCCS_ERR_INVALID_ARG;
+    return fused_common(ctx, Q, K, V, O, nullptr, key_len, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
 }
 
 hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
@@ -419,7 +429,7 @@ hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const i
                                        int32_t B, int32_t H, int32_t L, int32_t d,
                                        uint32_t flags, void *cuda_stream) {
     if (!out_scale) return HCCS_ERR_INVALID_ARG;
-    return fused_common(ctx, Q, K, V, O, out_scale, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+    return fused_common(ctx, Q, K, V, O, out_scale, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
 }
 
 hccs_status_t hccs_device_status(hccs_ctx_t *ctx, uint32_t *word, void *cuda_stream) {

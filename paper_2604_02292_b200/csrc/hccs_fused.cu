@@ -420,6 +420,16 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             mbar_arrive(smem_u32(&bars.s_free[sb]));
         };
         int amax_carry = -(1 << 30), r1_carry = 0;           // first-round blocks of a tile taken ahead of it
+        // number of valid keys (always a prefix) of this thread's row in the tile of head slice bh_ that
+        // starts at query q0_
+        auto valid_keys = [&](int bh_, int q0_) -> int {
+            int n = a.L;
+            if (CAUSAL) {
+                if (causal) n = min(q0_ + t + 1, n);
+                if (a.key_len) n = min(n, max(a.key_len[bh_ / a.H], 0));
+            }
+            return n;
+        };
 
         for (int tile = blockIdx.x, it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
             const int bh = tile / nblk, qt = tile % nblk;
@@ -430,9 +440,9 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head);   // host-prepared constants
             const float out_scale = __int_as_float(a.requant_mult[8 * head + 4]);
             const double inv_m = *reinterpret_cast<const double *>(a.requant_mult + 8 * head + 6);   // 1 / M_h
-            // valid keys of this row: all L of them, or the causal prefix (keys at and beyond L exist
-            // only as padding of the last block when L is no multiple of 128)
-            const int nv = (CAUSAL && causal) ? min(q0 + t + 1, a.L) : a.L;
+            // valid keys of this row: all L of them, the causal prefix, the batch entry's key length
+            // (keys at and beyond L exist only as padding of the last block when L is no multiple of 128)
+            const int nv = valid_keys(bh, q0);
 
             // the previous tile's O rows were staged in the panel: their bulk copies must have
             // read them before the panel is written again
@@ -632,7 +642,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if (two_rounds && tile + (int)gridDim.x < num_tiles) {
                 const int qt_n = (tile + (int)gridDim.x) % nblk;
                 const int kblocks_n = (CAUSAL && causal) ? qt_n + 1 : nblk;
-                const int nv_n = (CAUSAL && causal) ? min(qt_n * kTile + t + 1, a.L) : a.L;
+                const int nv_n = valid_keys((tile + (int)gridDim.x) / nblk, qt_n * kTile);
                 for (; ok && r1_carry < min(2, kblocks_n); ++r1_carry) first_round_block(r1_carry, nv_n, amax_carry);
             }
 
@@ -769,7 +779,9 @@ cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *laun
         return cudaErrorInvalidValue;
     cudaError_t e;
     // the masked instantiation also serves L that is no multiple of 128 (padding keys in the last block)
-    const bool clb = (a.flags & HCCS_RECIP_CLB) != 0, causal = (a.flags & HCCS_CAUSAL) != 0 || a.L % kTile != 0;
+    // and per-batch key lengths
+    const bool clb = (a.flags & HCCS_RECIP_CLB) != 0,
+               causal = (a.flags & HCCS_CAUSAL) != 0 || a.L % kTile != 0 || a.key_len != nullptr;
     if (a.d == 64) {
         if (!clb && !causal) e = launch_variant<64, false, false>(mq, mk, mv, mo, a, stream);
         else if (clb && !causal) e = launch_variant<64, true, false>(mq, mk, mv, mo, a, stream);

@@ -50,6 +50,7 @@ struct FusedArgs {
     const HeadEntry *table;
     const int32_t *requant_mult;   // device, 8 words per head: see fused_common in hccs_api.cu
     int32_t out_f32;               // 1: O = float(acc) * scale_h
+    const int32_t *key_len;        // device, one entry per batch entry, or NULL: keys beyond key_len[b] are padding
     uint32_t *status;
     int32_t requant_shift;
     int32_t B, H, L, d;
