@@ -159,24 +159,24 @@ def test_fp32_dequantised_output(hccs, oracle, d):
 
 
 @pytest.mark.parametrize("d,L", [(64, 1024), (64, 300), (128, 512)])
-@pytest.mark.parametrize("flags", [0, 4])
-def test_key_length_mask(hccs, oracle, d, L, flags):
+@pytest.mark.parametrize("flags,sh", [(0, 20), (4, 20), (0, 27), (6, 26)])
+def test_key_length_mask(hccs, oracle, d, L, flags, sh):
     """hccs_attention_fused_keylen: per-batch key lengths (0, 1, a block edge, ragged, L and beyond L),
     alone and with the causal rule."""
     import torch
-    rng = np.random.default_rng(6000 + d + L + flags)
+    rng = np.random.default_rng(6000 + d + L + flags + sh)
     Bt, H = 7, 2
     Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
     theta = hccs.workloads.sample_theta(rng, H, L)
-    mult = rng.integers(300, 1200, size=H).astype(np.int32)
+    mult = rng.integers(300, 1200, size=H).astype(np.int32) * (6 if sh > 24 else 1)
     key_len = np.array([0, 1, 128, min(L, 257), L - 1, L, L + 50], dtype=np.int32)
     ctx = hccs.Context(0)
     ctx.hccs_params_upload(theta, L)
     dQ, dK, dV = (torch.from_numpy(a).cuda() for a in (Q, K, V))
     O = torch.full(Q.shape, 0x7EADBEEF, dtype=torch.int32, device="cuda")
-    ctx.hccs_attention_fused_keylen(dQ, dK, dV, O, torch.from_numpy(key_len).cuda(), mult, 20, flags)
+    ctx.hccs_attention_fused_keylen(dQ, dK, dV, O, torch.from_numpy(key_len).cuda(), mult, sh, flags)
     torch.cuda.synchronize()
     assert ctx.hccs_device_status() == 0
-    want = oracle.attention(Q, K, V, mult, 20, theta, oracle_mode(oracle, flags), threads=16, key_len=key_len)
-    assert_same(O.cpu().numpy(), want, f"fused key_len d={d} L={L} flags={flags}")
+    want = oracle.attention(Q, K, V, mult, sh, theta, oracle_mode(oracle, flags), threads=16, key_len=key_len)
+    assert_same(O.cpu().numpy(), want, f"fused key_len d={d} L={L} flags={flags} sh={sh}")
     ctx.close()
