@@ -166,8 +166,8 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
  * hccs_attention_fused with a key-padding mask: key_len is a DEVICE int32 [B] array; keys at and
  * beyond key_len[b] (clamped to 0..L) of batch entry b are padding: like causally masked keys they
  * take no part in the row maximum and the row sum and get probability 0, so O is the attention over
- * the first key_len[b] keys alone; a batch entry with key length 0 gets O = 0.  Combines with
- * HCCS_CAUSAL.  Everything else as hccs_attention_fused.  (Masking is not in the paper, whose
+ * the first key_len[b] keys alone; a batch entry with key length 0 gets O = 0.  Key blocks that
+ * hold padding only are not computed at all.  Combines with HCCS_CAUSAL.  Everything else as hccs_attention_fused.  (Masking is not in the paper, whose
  * encoder workloads are padded to a fixed length, Section "Models and tasks".)
  */
 hccs_status_t hccs_attention_fused_keylen(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,

@@ -251,6 +251,19 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     tcgen05_fence_after();
     const uint32_t tmem = tmem_base_slot;
 
+    // Key blocks a tile goes through: all of the head's, or only those that hold a valid key for some row
+    // of the tile (causal rule, per-batch key length); at least one, so that O is written.
+    auto blocks_of = [&](int tile) -> int {
+        int n = nblk;
+        if (CAUSAL) {
+            if (causal) n = tile % nblk + 1;
+            if (a.key_len) {
+                const int kl = min(max(a.key_len[tile / nblk / a.H], 0), a.L);
+                n = min(n, max((kl + kTile - 1) / kTile, 1));
+            }
+        }
+        return n;
+    };
     // A CTA walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every mbarrier completes
     // one phase per use, so both sides count their uses (per barrier, because a causal tile uses
     // only its first qt + 1 key blocks) and wait on the parity of that count.
@@ -271,7 +284,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             };
             auto prefetch = [&](int tile) {
                 const int bh = tile / nblk, qt = tile % nblk;
-                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+                const int kblocks = blocks_of(tile);
                 load_tile(s_q, &map_q, bh * a.L + qt * kTile, smem_u32(&bars.q_full));
                 for (int kb = 0; kb < min(2, kblocks); ++kb) {
                     load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
@@ -279,8 +292,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             };
             if (me == 0 && (int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                const int bh = tile / nblk, qt = tile % nblk;
-                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+                const int bh = tile / nblk;
+                const int kblocks = blocks_of(tile);
                 // the other K blocks land where the previous tile's V sits: wait for its last MMA
                 if (it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (it - 1) & 1, abortp, a.status);
                 if (!ok) break;
@@ -315,8 +328,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const uint32_t dq_lo = (uint32_t)dq, dq_hi = (uint32_t)(dq >> 32);
             const uint32_t dk_lo = (uint32_t)dk, dk_hi = (uint32_t)(dk >> 32);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                const int qt = tile % nblk;
-                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+                const int kblocks = blocks_of(tile);
                 ok = mbar_wait(smem_u32(&bars.q_full), it & 1, abortp, a.status);
                 // the scan flow of the row warps reads every S block twice: once for the row maximum,
                 // once to requantise
@@ -365,8 +377,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const uint32_t dp_lo = (uint32_t)dp, dp_hi = (uint32_t)(dp >> 32);
             const uint32_t dv_lo = (uint32_t)dv, dv_hi = (uint32_t)(dv >> 32);
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int qt = tile % nblk;
-                const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+                const int kblocks = blocks_of(tile);
 #pragma unroll
                 for (int kb = 0; kb < kMaxBlocks; ++kb) {
                     if (kb >= kblocks) break;
@@ -435,7 +446,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int bh = tile / nblk, qt = tile % nblk;
             const int head = bh % a.H;
             const int q0 = qt * kTile;
-            const int kblocks = (CAUSAL && causal) ? qt + 1 : nblk;
+            const int kblocks = blocks_of(tile);
             const HeadEntry th = a.table[head];
             const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head);   // host-prepared constants
             const float out_scale = __int_as_float(a.requant_mult[8 * head + 4]);
@@ -641,7 +652,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             r1_carry = 0;
             if (two_rounds && tile + (int)gridDim.x < num_tiles) {
                 const int qt_n = (tile + (int)gridDim.x) % nblk;
-                const int kblocks_n = (CAUSAL && causal) ? qt_n + 1 : nblk;
+                const int kblocks_n = blocks_of(tile + (int)gridDim.x);
                 const int nv_n = valid_keys((tile + (int)gridDim.x) / nblk, qt_n * kTile);
                 for (; ok && r1_carry < min(2, kblocks_n); ++r1_carry) first_round_block(r1_carry, nv_n, amax_carry);
             }
