@@ -1,5 +1,5 @@
 // Register-resident row kernel for Lk = 32*G*V (G lanes per row, V 32-byte chunks per lane):
-// Lk = 32, 64, 128, ..., 2048.  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
+// Lk = 32, 64, 128, ..., 4096.  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
 //
 // Why 16-bit pairs: on sm_100a the byte-wise SIMD min/max intrinsics are emulated (about ten
 // instructions each), while min/max on s16x2 and the three-operand forms max(a+b, c) are single
@@ -272,6 +272,7 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
         case 512: return launch_gv<8, 2, U16, CLB, CAUSAL>(x, p, a, st);
         case 1024: return launch_gv<16, 2, U16, CLB, CAUSAL>(x, p, a, st);
         case 2048: return launch_gv<32, 2, U16, CLB, CAUSAL>(x, p, a, st);
+        case 4096: return launch_gv<32, 4, U16, CLB, CAUSAL>(x, p, a, st);
         default: break;
     }
     *taken = false;
