@@ -1,5 +1,5 @@
 // Register-resident row kernel for Lk = 32*G*V (G lanes per row, V 32-byte chunks per lane):
-// Lk = 32, 64, 128, ..., 4096.  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
+// the powers of two from 32 to 4096 and the multiples of 32 below 4096 whose odd part is 3, 5 or 7.  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
 //
 // Why 16-bit pairs: on sm_100a the byte-wise SIMD min/max intrinsics are emulated (about ten
 // instructions each), while min/max on s16x2 and the three-operand forms max(a+b, c) are single
@@ -273,6 +273,23 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
         case 1024: return launch_gv<16, 2, U16, CLB, CAUSAL>(x, p, a, st);
         case 2048: return launch_gv<32, 2, U16, CLB, CAUSAL>(x, p, a, st);
         case 4096: return launch_gv<32, 4, U16, CLB, CAUSAL>(x, p, a, st);
+        // three, five or seven 32-byte chunks per lane: the multiples of 32 whose odd part is 3, 5 or 7
+        case 96: return launch_gv<1, 3, U16, CLB, CAUSAL>(x, p, a, st);
+        case 192: return launch_gv<2, 3, U16, CLB, CAUSAL>(x, p, a, st);
+        case 384: return launch_gv<4, 3, U16, CLB, CAUSAL>(x, p, a, st);
+        case 768: return launch_gv<8, 3, U16, CLB, CAUSAL>(x, p, a, st);
+        case 1536: return launch_gv<16, 3, U16, CLB, CAUSAL>(x, p, a, st);
+        case 3072: return launch_gv<32, 3, U16, CLB, CAUSAL>(x, p, a, st);
+        case 160: return launch_gv<1, 5, U16, CLB, CAUSAL>(x, p, a, st);
+        case 320: return launch_gv<2, 5, U16, CLB, CAUSAL>(x, p, a, st);
+        case 640: return launch_gv<4, 5, U16, CLB, CAUSAL>(x, p, a, st);
+        case 1280: return launch_gv<8, 5, U16, CLB, CAUSAL>(x, p, a, st);
+        case 2560: return launch_gv<16, 5, U16, CLB, CAUSAL>(x, p, a, st);
+        case 224: return launch_gv<1, 7, U16, CLB, CAUSAL>(x, p, a, st);
+        case 448: return launch_gv<2, 7, U16, CLB, CAUSAL>(x, p, a, st);
+        case 896: return launch_gv<4, 7, U16, CLB, CAUSAL>(x, p, a, st);
+        case 1792: return launch_gv<8, 7, U16, CLB, CAUSAL>(x, p, a, st);
+        case 3584: return launch_gv<16, 7, U16, CLB, CAUSAL>(x, p, a, st);
         default: break;
     }
     *taken = false;

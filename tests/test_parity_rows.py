@@ -52,6 +52,19 @@ def test_row_lengths(ctx, oracle, hccs, Lk):
         _check(ctx, oracle, wl, flags)
 
 
+# the register-resident kernel's shapes with three, five or seven chunks per lane (and 4096 keys)
+@pytest.mark.parametrize("Lk", [96, 160, 192, 224, 320, 384, 448, 640, 768, 896, 1280, 1536, 1792, 2560,
+                                3072, 3584, 4096])
+@pytest.mark.parametrize("flags", ALL_FLAGS)
+def test_odd_chunk_counts(ctx, oracle, hccs, Lk, flags):
+    Lq = 70 if flags & 4 else 37                       # several warps, a ragged last warp, causal rows of every length class
+    wl = hccs.workloads.make_rows(7000 + Lk + flags, (2, 3, Lq, Lk), kind="gauss")
+    _check(ctx, oracle, wl, flags)
+    if flags & 4:                                      # square causal heads as well: every chunk-skipping case
+        wl = hccs.workloads.make_rows(7100 + Lk, (1, 2, min(Lk, 512), Lk), kind="laplace")
+        _check(ctx, oracle, wl, flags)
+
+
 @pytest.mark.parametrize("Lq,Lk", [(1, 64), (5, 64), (64, 5), (100, 128), (128, 100), (33, 512),
                                    (40, 1024), (7, 2048), (3, 1), (130, 144), (2100, 2048), (300, 4096),
                                    (4100, 4112)])
@@ -138,7 +151,7 @@ def test_every_row_sum_is_reached(ctx, oracle, hccs):
     assert set(range(383, 32705)) <= reached
 
 
-@pytest.mark.parametrize("Lk", [16, 33, 64, 128, 176, 512, 1024, 2048, 4096])
+@pytest.mark.parametrize("Lk", [16, 33, 64, 128, 160, 176, 512, 768, 1024, 2048, 4096])
 def test_key_length_mask(ctx, oracle, hccs, Lk):
     """hccs_forward_keylen: the padding mask of encoder workloads, alone and with the causal rule."""
     import torch
