@@ -64,6 +64,9 @@ cudaError_t launch_rows(const int8_t *logits, void *probs, const RowArgs &a, uin
 // Register-resident split-lane kernel (hccs_rows_split.cu): *taken tells whether the shape fit.
 cudaError_t try_launch_split(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                              cudaStream_t stream, bool *taken);
+// Span kernel for any row length up to 1024 keys and any alignment (hccs_rows_span.cu).
+cudaError_t try_launch_span(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                            cudaStream_t stream, bool *taken);
 // CTA-per-row kernel for long rows (hccs_rows_cta.cu).
 cudaError_t try_launch_cta(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                            cudaStream_t stream, bool *taken);

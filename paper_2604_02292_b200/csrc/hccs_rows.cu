@@ -8,6 +8,8 @@
 //                          owns a row, each lane holds V 16-byte vectors of it in registers.
 //   rows_cta_kernel        (hccs_rows_cta.cu) longer rows with Lk % 16 == 0: one CTA per row, the
 //                          row staged in shared memory by bulk asynchronous copies (TMA).
+//   rows_span_kernel       (hccs_rows_span.cu) any other Lk up to 1024 and any alignment: runs of rows
+//                          moved through shared memory as contiguous spans.
 //   rows_generic_kernel    everything else (any Lk, any alignment): one warp per row, bytes.
 //
 // Word-parallel identities used by the fast kernels (all exact):
@@ -275,6 +277,11 @@ cudaError_t launch_mode(const int8_t *x, void *p, const RowArgs &a, cudaStream_t
         if (taken) return e;
     }
     if (aligned && shift_ok && a.Lk <= 1024) return launch_lanegroup<U16, CLB, CAUSAL>(x, p, a, st);
+    if (shift_ok && a.Lk <= 1024) {         // any other length or alignment: rows moved as contiguous spans
+        bool taken = false;
+        cudaError_t e = try_launch_span(x, p, a, (U16 ? 1u : 0u) | (CLB ? 2u : 0u) | (CAUSAL ? 4u : 0u), st, &taken);
+        if (taken) return e;
+    }
     if (aligned) {
         bool taken = false;
         cudaError_t e = try_launch_cta(x, p, a, (U16 ? 1u : 0u) | (CLB ? 2u : 0u) | (CAUSAL ? 4u : 0u), st,

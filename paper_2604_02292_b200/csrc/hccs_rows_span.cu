@@ -1,0 +1,244 @@
+// Row kernel for any row length up to 1024 keys and any alignment of the tensors: rows whose
+// length is no multiple of 32 bytes cannot be fetched by the register-resident kernel with one
+// aligned vector load per lane, because a row then starts at an arbitrary byte.
+//
+// A CTA takes a run of consecutive rows -- one contiguous span of bytes, rows being back to back --
+// and moves it as a span: aligned 16-byte loads of the span's interior into shared memory (the
+// few bytes before the first and after the last 16-byte boundary go one by one), the rows are
+// worked on from shared memory, the results are laid down in a second span in shared memory and
+// leave it the same way.  Global memory traffic is therefore coalesced whatever Lk is.
+//
+// Inside the CTA G lanes own a row (G a power of two, 8 words of four keys per lane): a lane
+// assembles each of its words from the two aligned shared-memory words that hold it (the row
+// starts at an arbitrary byte), and from there Algorithm 1 runs on 16-bit pairs exactly as in
+// the register-resident kernel: stage 1 row max, stages 2-4 closeness r = max(x + (D - m), 0)
+// and its sum, stage 5 one reciprocal per row and p = (F*rho' + S*rho'*r) >> 16.  Word slots and
+// bytes beyond the row's valid keys (row end, causal rule, key length) are set to -128, can
+// then never raise the max, and their closeness is taken out of the sum in closed form.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hccs_device.cuh"
+#include "hccs_internal.h"
+
+namespace hccs {
+
+namespace {
+
+constexpr int kSpanThreads = 256;
+constexpr int kWordsPerLane = 8;
+constexpr uint32_t kMinus128x4 = 0x80808080u;
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
+    uint64_t d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t prefix_mask(int nbytes) {        // low nbytes bytes set (0..4, clamped)
+    return nbytes >= 4 ? 0xffffffffu : (nbytes <= 0 ? 0u : (1u << (8 * nbytes)) - 1u);
+}
+
+// Copies `bytes` bytes between global and shared memory; the two addresses are congruent modulo 16,
+// so the interior moves as aligned 16-byte vectors.  TO_SHARED: global -> shared, else shared -> global.
+template <bool TO_SHARED>
+__device__ __forceinline__ void copy_span(uint8_t *sm, uint8_t *gm, int64_t bytes) {
+    const int head = (int)min((int64_t)((16 - ((uintptr_t)gm & 15)) & 15), bytes);
+    const int64_t nvec = (bytes - head) >> 4;
+    const int tail = (int)(bytes - head - (nvec << 4));
+    for (int64_t v = threadIdx.x; v < nvec; v += kSpanThreads) {
+        uint4 *s = reinterpret_cast<uint4 *>(sm + head + (v << 4));
+        uint4 *g = reinterpret_cast<uint4 *>(gm + head + (v << 4));
+        if (TO_SHARED) *s = *g; else *g = *s;
+    }
+    const int edge = (int)threadIdx.x;
+    if (edge < head) { if (TO_SHARED) sm[edge] = gm[edge]; else gm[edge] = sm[edge]; }
+    if (edge >= 32 && edge - 32 < tail) {
+        const int64_t o = head + (nvec << 4) + (edge - 32);
+        if (TO_SHARED) sm[o] = gm[o]; else gm[o] = sm[o];
+    }
+}
+
+template <bool U16, bool CLB, bool MASKED>
+__global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x_all, void *p_all, RowArgs a,
+                                                                  int rows_per_cta, int log2_g) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    constexpr int OSZ = U16 ? 2 : 1;
+    const int Lk = a.Lk;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
+    const int nr = (int)min((int64_t)rows_per_cta, (int64_t)a.rows - r0);
+    const int64_t in_bytes = (int64_t)nr * Lk, out_bytes = in_bytes * OSZ;
+    uint8_t *g_in = const_cast<uint8_t *>(reinterpret_cast<const uint8_t *>(x_all)) + r0 * Lk;
+    uint8_t *g_out = reinterpret_cast<uint8_t *>(p_all) + r0 * Lk * OSZ;
+    // shared-memory images start at the same offset modulo 16 as their global spans
+    const int mis_in = (int)((uintptr_t)g_in & 15), mis_out = (int)((uintptr_t)g_out & 15);
+    const int in_room = (rows_per_cta * Lk + 47) & ~15;             // image + misalignment + one word of slack
+    uint8_t *s_in = smem + mis_in;
+    uint8_t *s_out = smem + in_room + mis_out;
+
+    copy_span<true>(s_in, g_in, in_bytes);
+    __syncthreads();
+
+    const int G = 1 << log2_g;
+    const int sub = threadIdx.x & (G - 1);
+    const int groups = kSpanThreads >> log2_g;                        // rows worked on at once
+    const int W = (Lk + 3) >> 2;                                      // words of a row, the last one maybe partial
+    const uint32_t *s_in_w = reinterpret_cast<const uint32_t *>(smem);
+    for (int i0 = 0; i0 < nr; i0 += groups) {                         // same trip count for every thread
+        const int i = i0 + (threadIdx.x >> log2_g);
+        const bool live = i < nr;
+        uint32_t bidx = 0, head = 0, qi = 0;
+        if (live) row_coords((uint32_t)(r0 + i), a, bidx, head, qi);
+        const int nv = live ? valid_keys<MASKED>(bidx, qi, a) : 0;
+        const HeadEntry th = a.table[head];
+
+        // ---- the lane's words: word j of the row lies at byte mis_in + i*Lk + 4j of the image
+        const int rb = mis_in + i * Lk;
+        const uint32_t sel = 0x3210u + 0x1111u * (uint32_t)(rb & 3);
+        uint32_t e[kWordsPerLane], o[kWordsPerLane];
+        uint32_t M = 0x80008000u;
+#pragma unroll
+        for (int k = 0; k < kWordsPerLane; ++k) {
+            const int j = sub + (k << log2_g);
+            uint32_t w = kMinus128x4;
+            if (live && j < W && 4 * j < nv) {
+                const int wi = (rb >> 2) + j;
+                w = prmt(s_in_w[wi], s_in_w[wi + 1], sel);
+                const uint32_t bm = prefix_mask(nv - 4 * j);
+                w = (w & bm) | (kMinus128x4 & ~bm);
+            }
+            const uint32_t ev = prmt(w, 0, 0xA280u), od = prmt(w, 0, 0xB391u);
+            e[k] = ev;
+            o[k] = od;
+            M = __vimax3_s16x2(M, ev, od);
+        }
+        int m = max((int)(short)(M & 0xffffu), (int)M >> 16);
+        for (int s = G >> 1; s; s >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, s));
+
+        // ---- closeness and its sum; every slot that holds no valid key was counted at x = -128
+        const int cm = th.D - m;
+        const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);
+        uint32_t rsum2 = 0;
+#pragma unroll
+        for (int k = 0; k < kWordsPerLane; ++k) {
+            e[k] = __viaddmax_s16x2(e[k], c2, 0u);
+            o[k] = __viaddmax_s16x2(o[k], c2, 0u);
+            rsum2 = rsum2 + e[k] + o[k];
+        }
+        int rsum = (int)(rsum2 & 0xffffu) + (int)(rsum2 >> 16);
+        for (int s = G >> 1; s; s >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, s);
+        rsum -= (4 * kWordsPerLane * G - nv) * max(cm - 128, 0);
+        const int F = th.B - th.S * th.D;
+        const uint32_t Z = (uint32_t)(nv * F + th.S * rsum);
+        const uint32_t rho = reciprocal<U16, CLB>(max(Z, 1u));
+        if (!live) continue;
+
+        // ---- normalise into the output image (rows start at arbitrary bytes there too)
+        uint8_t *orow = s_out + (int64_t)i * Lk * OSZ;
+        if (U16) {
+            const uint32_t a1 = (uint32_t)F * rho * 0x00010001u, b1 = (uint32_t)th.S * rho;
+#pragma unroll
+            for (int k = 0; k < kWordsPerLane; ++k) {
+                const int j = sub + (k << log2_g);
+                if (j >= W) continue;
+                const uint32_t pe = e[k] * b1 + a1, po = o[k] * b1 + a1;   // (p0, p2) and (p1, p3) as 16-bit pairs
+                uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
+                const uint32_t bm = prefix_mask(nv - 4 * j);
+                q0 &= prmt(bm, 0, 0x1100u);
+                q1 &= prmt(bm, 0, 0x3322u);
+                uint16_t *dst = reinterpret_cast<uint16_t *>(orow + 8 * j);      // 2-byte aligned: Lk*2 and mis_out even?
+                const int left = Lk - 4 * j;                                      // keys of the row from this word on
+                if (((uintptr_t)dst & 1) == 0) {
+                    dst[0] = (uint16_t)q0;
+                    if (left > 1) dst[1] = (uint16_t)(q0 >> 16);
+                    if (left > 2) dst[2] = (uint16_t)q1;
+                    if (left > 3) dst[3] = (uint16_t)(q1 >> 16);
+                } else {
+                    uint8_t *d8 = orow + 8 * j;
+                    const uint32_t qq[2] = {q0, q1};
+                    for (int b = 0; b < 8 && b < 2 * left; ++b) d8[b] = (uint8_t)(qq[b >> 2] >> (8 * (b & 3)));
+                }
+            }
+        } else {
+            const int sh = 1 - a.out_shift;                        // 0 or 1 (checked by the launcher)
+            const uint32_t rp = rho << sh;
+            const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+#pragma unroll
+            for (int k = 0; k < kWordsPerLane; ++k) {
+                const int j = sub + (k << log2_g);
+                if (j >= W) continue;
+                uint32_t q;
+                if (!CLB) {
+                    const uint64_t pe = mad_wide(prmt(e[k], 0, 0x2440u), b1, A);
+                    const uint64_t po = mad_wide(prmt(o[k], 0, 0x2440u), b1, A);
+                    q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                } else {
+                    const uint32_t x0 = min(a1 + b1 * (e[k] & 0xffffu), 0x00ffffffu);
+                    const uint32_t x1 = min(a1 + b1 * (o[k] & 0xffffu), 0x00ffffffu);
+                    const uint32_t x2 = min(a1 + b1 * (e[k] >> 16), 0x00ffffffu);
+                    const uint32_t x3 = min(a1 + b1 * (o[k] >> 16), 0x00ffffffu);
+                    q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                }
+                q &= prefix_mask(nv - 4 * j);
+                uint8_t *dst = orow + 4 * j;
+                const int left = Lk - 4 * j;
+                if (((uintptr_t)dst & 3) == 0 && left >= 4) {
+                    *reinterpret_cast<uint32_t *>(dst) = q;
+                } else {
+                    dst[0] = (uint8_t)q;
+                    if (left > 1) dst[1] = (uint8_t)(q >> 8);
+                    if (left > 2) dst[2] = (uint8_t)(q >> 16);
+                    if (left > 3) dst[3] = (uint8_t)(q >> 24);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    copy_span<false>(s_out, g_out, out_bytes);
+}
+
+template <bool U16, bool CLB, bool MASKED>
+cudaError_t launch_span(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
+    constexpr int OSZ = U16 ? 2 : 1;
+    // 8 words per lane: the smallest power of two of lanes that covers the row
+    const int W = (a.Lk + 3) / 4;
+    int log2_g = 0;
+    while ((kWordsPerLane << log2_g) < W) ++log2_g;
+    // rows per CTA: both images within 48 KB of shared memory, at most four passes of all lane groups
+    const int budget = 47 * 1024 - 64;
+    int rows_per_cta = budget / (a.Lk * (1 + OSZ));
+    const int groups = kSpanThreads >> log2_g;
+    if (rows_per_cta > 4 * groups) rows_per_cta = 4 * groups;
+    if (rows_per_cta < 1) rows_per_cta = 1;
+    const size_t smem = (size_t)((rows_per_cta * a.Lk + 47) & ~15) + (size_t)((rows_per_cta * a.Lk * OSZ + 31) & ~15) + 16;
+    const unsigned blocks = (unsigned)(((int64_t)a.rows + rows_per_cta - 1) / rows_per_cta);
+    rows_span_kernel<U16, CLB, MASKED><<<blocks, kSpanThreads, smem, st>>>(x, p, a, rows_per_cta, log2_g);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t try_launch_span(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
+                            cudaStream_t stream, bool *taken) {
+    *taken = false;
+    if (a.Lk < 1 || a.Lk > 4 * kWordsPerLane * 32) return cudaSuccess;     // 1024 keys at most
+    if (!(flags & 1u) && a.out_shift > 1) return cudaSuccess;
+    *taken = true;
+    switch (flags & 7u) {
+        case 0: return launch_span<false, false, false>(logits, probs, a, stream);
+        case 1: return launch_span<true, false, false>(logits, probs, a, stream);
+        case 2: return launch_span<false, true, false>(logits, probs, a, stream);
+        case 3: return launch_span<true, true, false>(logits, probs, a, stream);
+        case 4: return launch_span<false, false, true>(logits, probs, a, stream);
+        case 5: return launch_span<true, false, true>(logits, probs, a, stream);
+        case 6: return launch_span<false, true, true>(logits, probs, a, stream);
+        default: return launch_span<true, true, true>(logits, probs, a, stream);
+    }
+}
+
+}  // namespace hccs
