@@ -96,25 +96,32 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
         const int nv = live ? valid_keys<MASKED>(bidx, qi, a) : 0;
         const HeadEntry th = a.table[head];
 
-        // ---- the lane's words: word j of the row lies at byte mis_in + i*Lk + 4j of the image
+        // ---- the lane's words: word j of the row lies at byte mis_in + i*Lk + 4j of the image.
+        // valid bytes of word j: min(nv - 4j, 4); without a mask only the row's last word can be partial
         const int rb = mis_in + i * Lk;
         const uint32_t sel = 0x3210u + 0x1111u * (uint32_t)(rb & 3);
+        const uint32_t tail_mask = prefix_mask(Lk - 4 * (W - 1));
+        auto word_mask = [&](int j) -> uint32_t {
+            if (MASKED) return __funnelshift_rc(0xffffffffu, 0u, 32 - 8 * min(max(nv - 4 * j, 0), 4));
+            return j == W - 1 ? tail_mask : 0xffffffffu;
+        };
         uint32_t e[kWordsPerLane], o[kWordsPerLane];
         uint32_t M = 0x80008000u;
+        {
+            int j = sub, wi = (rb >> 2) + sub;
 #pragma unroll
-        for (int k = 0; k < kWordsPerLane; ++k) {
-            const int j = sub + (k << log2_g);
-            uint32_t w = kMinus128x4;
-            if (live && j < W && 4 * j < nv) {
-                const int wi = (rb >> 2) + j;
-                w = prmt(s_in_w[wi], s_in_w[wi + 1], sel);
-                const uint32_t bm = prefix_mask(nv - 4 * j);
-                w = (w & bm) | (kMinus128x4 & ~bm);
+            for (int k = 0; k < kWordsPerLane; ++k, j += G, wi += G) {
+                uint32_t w = kMinus128x4;
+                if (live && j < W && (!MASKED || 4 * j < nv)) {
+                    w = prmt(s_in_w[wi], s_in_w[wi + 1], sel);
+                    const uint32_t bm = word_mask(j);
+                    w = (w & bm) | (kMinus128x4 & ~bm);
+                }
+                const uint32_t ev = prmt(w, 0, 0xA280u), od = prmt(w, 0, 0xB391u);
+                e[k] = ev;
+                o[k] = od;
+                M = __vimax3_s16x2(M, ev, od);
             }
-            const uint32_t ev = prmt(w, 0, 0xA280u), od = prmt(w, 0, 0xB391u);
-            e[k] = ev;
-            o[k] = od;
-            M = __vimax3_s16x2(M, ev, od);
         }
         int m = max((int)(short)(M & 0xffffu), (int)M >> 16);
         for (int s = G >> 1; s; s >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, s));
@@ -137,30 +144,32 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
         const uint32_t rho = reciprocal<U16, CLB>(max(Z, 1u));
         if (!live) continue;
 
-        // ---- normalise into the output image (rows start at arbitrary bytes there too)
-        uint8_t *orow = s_out + (int64_t)i * Lk * OSZ;
+        // ---- normalise into the output image (rows start at arbitrary bytes there too): word j of the
+        // row goes to byte ob + 4j*OSZ of the shared-memory array; whole aligned words in one store
+        const int ob = in_room + mis_out + i * Lk * OSZ;
+        const bool row_aligned = (ob & 3) == 0;
         if (U16) {
             const uint32_t a1 = (uint32_t)F * rho * 0x00010001u, b1 = (uint32_t)th.S * rho;
+            int j = sub;
 #pragma unroll
-            for (int k = 0; k < kWordsPerLane; ++k) {
-                const int j = sub + (k << log2_g);
+            for (int k = 0; k < kWordsPerLane; ++k, j += G) {
                 if (j >= W) continue;
                 const uint32_t pe = e[k] * b1 + a1, po = o[k] * b1 + a1;   // (p0, p2) and (p1, p3) as 16-bit pairs
                 uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
-                const uint32_t bm = prefix_mask(nv - 4 * j);
+                const uint32_t bm = word_mask(j);
                 q0 &= prmt(bm, 0, 0x1100u);
                 q1 &= prmt(bm, 0, 0x3322u);
-                uint16_t *dst = reinterpret_cast<uint16_t *>(orow + 8 * j);      // 2-byte aligned: Lk*2 and mis_out even?
                 const int left = Lk - 4 * j;                                      // keys of the row from this word on
-                if (((uintptr_t)dst & 1) == 0) {
-                    dst[0] = (uint16_t)q0;
-                    if (left > 1) dst[1] = (uint16_t)(q0 >> 16);
-                    if (left > 2) dst[2] = (uint16_t)q1;
-                    if (left > 3) dst[3] = (uint16_t)(q1 >> 16);
+                uint8_t *dst = smem + ob + 8 * j;
+                if (row_aligned && left >= 4) {
+                    reinterpret_cast<uint32_t *>(dst)[0] = q0;
+                    reinterpret_cast<uint32_t *>(dst)[1] = q1;
                 } else {
-                    uint8_t *d8 = orow + 8 * j;
-                    const uint32_t qq[2] = {q0, q1};
-                    for (int b = 0; b < 8 && b < 2 * left; ++b) d8[b] = (uint8_t)(qq[b >> 2] >> (8 * (b & 3)));
+                    uint16_t *d16 = reinterpret_cast<uint16_t *>(dst);           // uint16 tensors are 2-byte aligned
+                    d16[0] = (uint16_t)q0;
+                    if (left > 1) d16[1] = (uint16_t)(q0 >> 16);
+                    if (left > 2) d16[2] = (uint16_t)q1;
+                    if (left > 3) d16[3] = (uint16_t)(q1 >> 16);
                 }
             }
         } else {
@@ -168,9 +177,9 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
             const uint32_t rp = rho << sh;
             const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
             const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+            int j = sub;
 #pragma unroll
-            for (int k = 0; k < kWordsPerLane; ++k) {
-                const int j = sub + (k << log2_g);
+            for (int k = 0; k < kWordsPerLane; ++k, j += G) {
                 if (j >= W) continue;
                 uint32_t q;
                 if (!CLB) {
@@ -184,10 +193,10 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
                     const uint32_t x3 = min(a1 + b1 * (o[k] >> 16), 0x00ffffffu);
                     q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
                 }
-                q &= prefix_mask(nv - 4 * j);
-                uint8_t *dst = orow + 4 * j;
+                q &= word_mask(j);
                 const int left = Lk - 4 * j;
-                if (((uintptr_t)dst & 3) == 0 && left >= 4) {
+                uint8_t *dst = smem + ob + 4 * j;
+                if (row_aligned && left >= 4) {
                     *reinterpret_cast<uint32_t *>(dst) = q;
                 } else {
                     dst[0] = (uint8_t)q;
