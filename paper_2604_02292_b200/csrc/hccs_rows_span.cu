@@ -8,7 +8,7 @@
 // worked on from shared memory, the results are laid down in a second span in shared memory and
 // leave it the same way.  Global memory traffic is therefore coalesced whatever Lk is.
 //
-// Inside the CTA G lanes own a row (G a power of two, 8 words of four keys per lane): a lane
+// Inside the CTA G lanes own a row (G a power of two, up to 8 words of four keys per lane): a lane
 // assembles each of its words from the two aligned shared-memory words that hold it (the row
 // starts at an arbitrary byte), and from there Algorithm 1 runs on 16-bit pairs exactly as in
 // the register-resident kernel: stage 1 row max, stages 2-4 closeness r = max(x + (D - m), 0)
@@ -26,7 +26,7 @@ namespace hccs {
 namespace {
 
 constexpr int kSpanThreads = 256;
-constexpr int kWordsPerLane = 8;
+constexpr int kMaxWordsPerLane = 8;
 constexpr uint32_t kMinus128x4 = 0x80808080u;
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
@@ -63,7 +63,7 @@ __device__ __forceinline__ void copy_span(uint8_t *sm, uint8_t *gm, int64_t byte
     }
 }
 
-template <bool U16, bool CLB, bool MASKED>
+template <int kWordsPerLane, bool U16, bool CLB, bool MASKED>
 __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x_all, void *p_all, RowArgs a,
                                                                   int rows_per_cta, int log2_g) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -211,13 +211,9 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
     copy_span<false>(s_out, g_out, out_bytes);
 }
 
-template <bool U16, bool CLB, bool MASKED>
-cudaError_t launch_span(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
+template <int WPL, bool U16, bool CLB, bool MASKED>
+cudaError_t launch_span_w(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st, int log2_g) {
     constexpr int OSZ = U16 ? 2 : 1;
-    // 8 words per lane: the smallest power of two of lanes that covers the row
-    const int W = (a.Lk + 3) / 4;
-    int log2_g = 0;
-    while ((kWordsPerLane << log2_g) < W) ++log2_g;
     // rows per CTA: both images within 48 KB of shared memory, at most four passes of all lane groups
     const int budget = 47 * 1024 - 64;
     int rows_per_cta = budget / (a.Lk * (1 + OSZ));
@@ -226,8 +222,28 @@ cudaError_t launch_span(const int8_t *x, void *p, const RowArgs &a, cudaStream_t
     if (rows_per_cta < 1) rows_per_cta = 1;
     const size_t smem = (size_t)((rows_per_cta * a.Lk + 47) & ~15) + (size_t)((rows_per_cta * a.Lk * OSZ + 31) & ~15) + 16;
     const unsigned blocks = (unsigned)(((int64_t)a.rows + rows_per_cta - 1) / rows_per_cta);
-    rows_span_kernel<U16, CLB, MASKED><<<blocks, kSpanThreads, smem, st>>>(x, p, a, rows_per_cta, log2_g);
+    rows_span_kernel<WPL, U16, CLB, MASKED><<<blocks, kSpanThreads, smem, st>>>(x, p, a, rows_per_cta, log2_g);
     return cudaGetLastError();
+}
+
+template <bool U16, bool CLB, bool MASKED>
+cudaError_t launch_span(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
+    // G lanes per row, the smallest power of two that covers the row's words with at most 8 per lane;
+    // then as few words per lane as cover it (the unused slots of a lane cost as much as the used ones)
+    const int W = (a.Lk + 3) / 4;
+    int log2_g = 0;
+    while ((kMaxWordsPerLane << log2_g) < W) ++log2_g;
+    const int wpl = (W + (1 << log2_g) - 1) >> log2_g;
+    switch (wpl) {
+        case 1: return launch_span_w<1, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        case 2: return launch_span_w<2, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        case 3: return launch_span_w<3, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        case 4: return launch_span_w<4, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        case 5: return launch_span_w<5, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        case 6: return launch_span_w<6, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        case 7: return launch_span_w<7, U16, CLB, MASKED>(x, p, a, st, log2_g);
+        default: return launch_span_w<8, U16, CLB, MASKED>(x, p, a, st, log2_g);
+    }
 }
 
 }  // namespace
@@ -235,7 +251,7 @@ cudaError_t launch_span(const int8_t *x, void *p, const RowArgs &a, cudaStream_t
 cudaError_t try_launch_span(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                             cudaStream_t stream, bool *taken) {
     *taken = false;
-    if (a.Lk < 1 || a.Lk > 4 * kWordsPerLane * 32) return cudaSuccess;     // 1024 keys at most
+    if (a.Lk < 1 || a.Lk > 4 * kMaxWordsPerLane * 32) return cudaSuccess;  // 1024 keys at most
     if (!(flags & 1u) && a.out_shift > 1) return cudaSuccess;
     *taken = true;
     switch (flags & 7u) {
