@@ -63,6 +63,27 @@ __device__ __forceinline__ void stg256(void *p, const uint32_t (&r)[8]) {
                  : "memory");
 }
 
+// The same for 16-byte chunks.
+template <bool EVICT_FIRST>
+__device__ __forceinline__ void ldg128(const void *p, uint32_t (&r)[4]) {
+    if (EVICT_FIRST) {
+        uint64_t pol;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+        asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                     : "l"(p), "l"(pol));
+    } else {
+        asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                     : "l"(p));
+    }
+}
+__device__ __forceinline__ void stg128(void *p, const uint32_t (&r)[4]) {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]),
+                 "r"(r[3])
+                 : "memory");
+}
+
 __device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
     uint64_t d;
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
@@ -74,14 +95,17 @@ constexpr uint32_t kSelOdd = 0xB391u;    // bytes 1 and 3, each sign-extended to
 constexpr uint32_t kSelWide = 0x2440u;   // 16-bit pair (r_a, r_b) -> r_a + r_b * 2^24
 constexpr uint32_t kMinus128x4 = 0x80808080u;
 
-template <int G, int V, bool U16, bool CLB, bool CAUSAL>
+// CW: 32-bit words per chunk, 8 (32-byte chunks) or 4 (16-byte chunks, for the row lengths that are a
+// multiple of 16 but not of 32, or whose number of 32-byte chunks has an odd part above 7).
+template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8>
 __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, void *p_all, RowArgs a) {
     constexpr int RW = 32 / G;      // rows per warp
-    constexpr int NW = 8 * V;       // 32-bit words of logits per lane
-    __shared__ uint32_t mask_tab[CAUSAL ? 33 * 8 : 1];   // [valid bytes of a chunk][word] -> byte mask
+    constexpr int NW = CW * V;      // 32-bit words of logits per lane
+    constexpr int CB = 4 * CW;      // bytes (keys) per chunk
+    __shared__ uint32_t mask_tab[CAUSAL ? (CB + 1) * CW : 1];   // [valid bytes of a chunk][word] -> byte mask
     if (CAUSAL) {
-        for (int idx = threadIdx.x; idx < 33 * 8; idx += blockDim.x) {
-            const int nb = idx / 8 - 4 * (idx % 8);
+        for (int idx = threadIdx.x; idx < (CB + 1) * CW; idx += blockDim.x) {
+            const int nb = idx / CW - 4 * (idx % CW);
             mask_tab[idx] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
         }
         __syncthreads();
@@ -103,11 +127,11 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     // Causal: a chunk index v whose columns lie beyond every row of this warp is skipped
     // altogether (warp-uniform), e.g. the right half of the first 64 queries of a 128-key head.
     const int warp_nv = CAUSAL ? __reduce_max_sync(0xffffffffu, nv) : a.Lk;
-    auto chunk_used = [&](int v) { return !CAUSAL || v == 0 || v * G * 32 < warp_nv; };
+    auto chunk_used = [&](int v) { return !CAUSAL || v == 0 || v * G * CB < warp_nv; };
     int skipped_cols = 0;           // masked columns of this row that were never materialised
 #pragma unroll
     for (int v = 1; v < V; ++v)
-        if (!chunk_used(v)) skipped_cols += 32 * G;
+        if (!chunk_used(v)) skipped_cols += CB * G;
 
     // ---- loads: V independent 32-byte requests per lane
     uint32_t e[NW], o[NW];          // first the raw words (in e), then the split lanes
@@ -115,17 +139,18 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     const int8_t *x_row = x_all + (int64_t)row * a.Lk;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-        const int col = (sub + v * G) * 32;
-        cnt[v] = CAUSAL ? min(max(nv - col, 0), 32) : (live ? 32 : 0);
-        uint32_t w[8];
+        const int col = (sub + v * G) * CB;
+        cnt[v] = CAUSAL ? min(max(nv - col, 0), CB) : (live ? CB : 0);
+        uint32_t w[CW];
         if (cnt[v] > 0) {
-            ldg256<G == 1>(x_row + col, w);
+            if constexpr (CW == 8) ldg256<G == 1>(x_row + col, w);
+            else ldg128<G == 1>(x_row + col, w);
         } else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) w[k] = kMinus128x4;
+            for (int k = 0; k < CW; ++k) w[k] = kMinus128x4;
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) e[8 * v + k] = w[k];
+        for (int k = 0; k < CW; ++k) e[CW * v + k] = w[k];
     }
 
     // ---- split into 16-bit lanes; stage 1: row max
@@ -134,15 +159,15 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     for (int v = 0; v < V; ++v) {
         if (!chunk_used(v)) continue;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            uint32_t w = e[8 * v + k];
+        for (int k = 0; k < CW; ++k) {
+            uint32_t w = e[CW * v + k];
             if (CAUSAL) {
-                const uint32_t bm = mask_tab[cnt[v] * 8 + k];
+                const uint32_t bm = mask_tab[cnt[v] * CW + k];
                 w = (w & bm) | (kMinus128x4 & ~bm);
             }
             const uint32_t ev = prmt(w, 0, kSelEven), od = prmt(w, 0, kSelOdd);
-            e[8 * v + k] = ev;
-            o[8 * v + k] = od;
+            e[CW * v + k] = ev;
+            o[CW * v + k] = od;
             M = __vimax3_s16x2(M, ev, od);
         }
     }
@@ -158,7 +183,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     for (int v = 0; v < V; ++v) {
         if (!chunk_used(v)) continue;
 #pragma unroll
-        for (int k = 8 * v; k < 8 * v + 8; ++k) {
+        for (int k = CW * v; k < CW * v + CW; ++k) {
             e[k] = __viaddmax_s16x2(e[k], c2, 0u);
             o[k] = __viaddmax_s16x2(o[k], c2, 0u);
             rsum2 = rsum2 + e[k] + o[k];                   // lane sums stay below 2^16
@@ -180,29 +205,33 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         uint16_t *p_row = (uint16_t *)p_all + (int64_t)row * a.Lk;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
-            const int col = (sub + v * G) * 32;
-            uint32_t out[16];
+            const int col = (sub + v * G) * CB;
+            uint32_t out[2 * CW];
             if (!chunk_used(v)) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k) out[k] = 0;
+                for (int k = 0; k < 2 * CW; ++k) out[k] = 0;
             } else
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t pe = e[8 * v + k] * b1 + a1, po = o[8 * v + k] * b1 + a1;
+            for (int k = 0; k < CW; ++k) {
+                const uint32_t pe = e[CW * v + k] * b1 + a1, po = o[CW * v + k] * b1 + a1;
                 uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
                 if (CAUSAL) {
-                    const uint32_t bm = mask_tab[cnt[v] * 8 + k];
+                    const uint32_t bm = mask_tab[cnt[v] * CW + k];
                     q0 &= prmt(bm, 0, 0x1100u);
                     q1 &= prmt(bm, 0, 0x3322u);
                 }
                 out[2 * k] = q0;
                 out[2 * k + 1] = q1;
             }
-            uint32_t lo[8], hi[8];
+            if constexpr (CW == 8) {
+                uint32_t lo[8], hi[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) { lo[k] = out[k]; hi[k] = out[8 + k]; }
-            stg256(p_row + col, lo);
-            stg256(p_row + col + 16, hi);
+                for (int k = 0; k < 8; ++k) { lo[k] = out[k]; hi[k] = out[8 + k]; }
+                stg256(p_row + col, lo);
+                stg256(p_row + col + 16, hi);
+            } else {
+                stg256(p_row + col, out);
+            }
         }
     } else {
         const int sh = 1 - a.out_shift;                    // 0 or 1 (checked by the launcher)
@@ -211,41 +240,42 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         uint8_t *p_row = (uint8_t *)p_all + (int64_t)row * a.Lk;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
-            const int col = (sub + v * G) * 32;
-            uint32_t out[8];
+            const int col = (sub + v * G) * CB;
+            uint32_t out[CW];
             if (!chunk_used(v)) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) out[k] = 0;
+                for (int k = 0; k < CW; ++k) out[k] = 0;
             } else
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < CW; ++k) {
                 uint32_t q;
                 if (!CLB) {
                     const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
-                    const uint64_t pe = mad_wide(prmt(e[8 * v + k], 0, kSelWide), b1, A);
-                    const uint64_t po = mad_wide(prmt(o[8 * v + k], 0, kSelWide), b1, A);
+                    const uint64_t pe = mad_wide(prmt(e[CW * v + k], 0, kSelWide), b1, A);
+                    const uint64_t po = mad_wide(prmt(o[CW * v + k], 0, kSelWide), b1, A);
                     // bytes 2,3 of the high words are zero: [p0,0,p2,0] + [0,p1,0,p3]
                     const uint32_t t0 = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u);
                     const uint32_t t1 = prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
                     q = t0 + t1;
                 } else {
                     // the leading-bit reciprocal can overshoot 255: saturate each element
-                    const uint32_t ev = e[8 * v + k], od = o[8 * v + k];
+                    const uint32_t ev = e[CW * v + k], od = o[CW * v + k];
                     const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
                     const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
                     const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
                     const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
                     q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
                 }
-                if (CAUSAL) q &= mask_tab[cnt[v] * 8 + k];
+                if (CAUSAL) q &= mask_tab[cnt[v] * CW + k];
                 out[k] = q;
             }
-            stg256(p_row + col, out);
+            if constexpr (CW == 8) stg256(p_row + col, out);
+            else stg128(p_row + col, out);
         }
     }
 }
 
-template <int G, int V, bool U16, bool CLB, bool CAUSAL>
+template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8>
 cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
     constexpr int ROWS_PER_CTA = 8 * (32 / G);
     const unsigned blocks = (unsigned)(((int64_t)a.rows + ROWS_PER_CTA - 1) / ROWS_PER_CTA);
@@ -258,7 +288,7 @@ cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL>, x, p, a);
+    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL, CW>, x, p, a);
 }
 
 template <bool U16, bool CLB, bool CAUSAL>
@@ -291,6 +321,21 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
         case 1792: return launch_gv<8, 7, U16, CLB, CAUSAL>(x, p, a, st);
         case 3584: return launch_gv<16, 7, U16, CLB, CAUSAL>(x, p, a, st);
         default: break;
+    }
+    // 16-byte chunks: Lk = 16 * G * V with V odd, 3 <= V <= 15 -- every multiple of 16 up to 7680 whose odd
+    // part is at most 15 and that the cases above do not take (48, 80, 112, 144, 176, ..., 288, 576, ...)
+    if (a.Lk % 16 == 0) {
+        int v = a.Lk / 16, g = 1;
+        while ((v & 1) == 0) { v >>= 1; g <<= 1; }
+        if (g <= 32 && v >= 3 && v <= 15) {
+#define HCCS_SPLIT16(GG, VV) if (g == GG && v == VV) return launch_gv<GG, VV, U16, CLB, CAUSAL, 4>(x, p, a, st);
+#define HCCS_SPLIT16_G(VV) HCCS_SPLIT16(1, VV) HCCS_SPLIT16(2, VV) HCCS_SPLIT16(4, VV) HCCS_SPLIT16(8, VV) \
+                           HCCS_SPLIT16(16, VV) HCCS_SPLIT16(32, VV)
+            HCCS_SPLIT16_G(3) HCCS_SPLIT16_G(5) HCCS_SPLIT16_G(7) HCCS_SPLIT16_G(9) HCCS_SPLIT16_G(11)
+            HCCS_SPLIT16_G(13) HCCS_SPLIT16_G(15)
+#undef HCCS_SPLIT16_G
+#undef HCCS_SPLIT16
+        }
     }
     *taken = false;
     return cudaSuccess;

@@ -54,7 +54,10 @@ def test_row_lengths(ctx, oracle, hccs, Lk):
 
 # the register-resident kernel's shapes with three, five or seven chunks per lane (and 4096 keys)
 @pytest.mark.parametrize("Lk", [96, 160, 192, 224, 320, 384, 448, 640, 768, 896, 1280, 1536, 1792, 2560,
-                                3072, 3584, 4096])
+                                3072, 3584, 4096,
+                                # 16-byte chunks: multiples of 16 whose odd part is 3 ... 15
+                                48, 80, 112, 144, 176, 208, 240, 288, 352, 416, 480, 576, 960, 1152, 2304,
+                                3328, 4608, 7680])
 @pytest.mark.parametrize("flags", ALL_FLAGS)
 def test_odd_chunk_counts(ctx, oracle, hccs, Lk, flags):
     Lq = 70 if flags & 4 else 37                       # several warps, a ragged last warp, causal rows of every length class
