@@ -98,8 +98,11 @@ constexpr uint32_t kMinus128x4 = 0x80808080u;
 
 // CW: 32-bit words per chunk, 8 (32-byte chunks) or 4 (16-byte chunks, for the row lengths that are a
 // multiple of 16 but not of 32, or whose number of 32-byte chunks has an odd part above 7).
-template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8>
+// PAD: the G*V chunks of a lane group cover more than the row (any multiple of 16 keys: the chunks beyond
+// the row's end are never loaded, count as masked and are not stored); needs the masked instantiation.
+template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8, bool PAD = false>
 __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, void *p_all, RowArgs a) {
+    static_assert(!PAD || CAUSAL, "padded lane groups run through the masked path");
     constexpr int RW = 32 / G;      // rows per warp
     constexpr int NW = CW * V;      // 32-bit words of logits per lane
     constexpr int CB = 4 * CW;      // bytes (keys) per chunk
@@ -194,7 +197,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
 #pragma unroll
     for (int s = G / 2; s; s >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, s);
     // masked keys that were materialised were counted at x = -128
-    if (CAUSAL) rsum -= (a.Lk - nv - skipped_cols) * max(cm - 128, 0);
+    if (CAUSAL) rsum -= ((PAD ? G * V * CB : a.Lk) - nv - skipped_cols) * max(cm - 128, 0);
     const int F = th.B - th.S * th.D;                      // floor score
     const uint32_t Z = (uint32_t)(nv * F + th.S * rsum);
     const uint32_t rho = reciprocal<U16, CLB>(max(Z, 1u));
@@ -207,6 +210,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int col = (sub + v * G) * CB;
+            if (PAD && col >= a.Lk) continue;
             uint32_t out[2 * CW];
             if (!chunk_used(v)) {
 #pragma unroll
@@ -242,6 +246,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int col = (sub + v * G) * CB;
+            if (PAD && col >= a.Lk) continue;
             uint32_t out[CW];
             if (!chunk_used(v)) {
 #pragma unroll
@@ -276,7 +281,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     }
 }
 
-template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8>
+template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8, bool PAD = false>
 cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
     constexpr int ROWS_PER_CTA = 8 * (32 / G);
     const unsigned blocks = (unsigned)(((int64_t)a.rows + ROWS_PER_CTA - 1) / ROWS_PER_CTA);
@@ -289,7 +294,7 @@ cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL, CW>, x, p, a);
+    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL, CW, PAD>, x, p, a);
 }
 
 template <bool U16, bool CLB, bool CAUSAL>
@@ -336,6 +341,16 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
             HCCS_SPLIT16_G(13) HCCS_SPLIT16_G(15)
 #undef HCCS_SPLIT16_G
 #undef HCCS_SPLIT16
+        }
+        // every other multiple of 16 up to 4096: eight 16-byte chunks per lane, the smallest power of two
+        // of lanes that covers the row, the excess chunks padded (masked path, also without a mask)
+        const int chunks = a.Lk / 16;
+        if (chunks > 8 && chunks <= 8 * 32) {
+            if (chunks <= 16) return launch_gv<2, 8, U16, CLB, true, 4, true>(x, p, a, st);
+            if (chunks <= 32) return launch_gv<4, 8, U16, CLB, true, 4, true>(x, p, a, st);
+            if (chunks <= 64) return launch_gv<8, 8, U16, CLB, true, 4, true>(x, p, a, st);
+            if (chunks <= 128) return launch_gv<16, 8, U16, CLB, true, 4, true>(x, p, a, st);
+            return launch_gv<32, 8, U16, CLB, true, 4, true>(x, p, a, st);
         }
     }
     *taken = false;
