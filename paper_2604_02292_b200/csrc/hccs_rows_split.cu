@@ -1,5 +1,6 @@
 // Register-resident row kernel for Lk = 32*G*V (G lanes per row, V 32-byte chunks per lane):
-// the powers of two from 32 to 4096 and the multiples of 32 below 4096 whose odd part is 3, 5 or 7.  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
+// the powers of two from 32 to 8192 and the multiples of 32 below 4096 whose odd part is 3, 5 or 7
+// (and, with 16-byte chunks or padded lane groups, the other multiples of 16: see launch_shape).  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
 //
 // Why 16-bit pairs: on sm_100a the byte-wise SIMD min/max intrinsics are emulated (about ten
 // instructions each), while min/max on s16x2 and the three-operand forms max(a+b, c) are single
@@ -309,6 +310,7 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
         case 1024: return launch_gv<16, 2, U16, CLB, CAUSAL>(x, p, a, st);
         case 2048: return launch_gv<32, 2, U16, CLB, CAUSAL>(x, p, a, st);
         case 4096: return launch_gv<32, 4, U16, CLB, CAUSAL>(x, p, a, st);
+        case 8192: return launch_gv<32, 8, U16, CLB, CAUSAL>(x, p, a, st);
         // three, five or seven 32-byte chunks per lane: the multiples of 32 whose odd part is 3, 5 or 7
         case 96: return launch_gv<1, 3, U16, CLB, CAUSAL>(x, p, a, st);
         case 192: return launch_gv<2, 3, U16, CLB, CAUSAL>(x, p, a, st);
@@ -352,6 +354,8 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
             if (chunks <= 128) return launch_gv<16, 8, U16, CLB, true, 4, true>(x, p, a, st);
             return launch_gv<32, 8, U16, CLB, true, 4, true>(x, p, a, st);
         }
+        // ... and the multiples of 32 from there to 8192: eight 32-byte chunks per lane, a whole warp per row
+        if (a.Lk % 32 == 0 && a.Lk <= 8192) return launch_gv<32, 8, U16, CLB, true, 8, true>(x, p, a, st);
     }
     *taken = false;
     return cudaSuccess;

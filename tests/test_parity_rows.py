@@ -59,7 +59,8 @@ def test_row_lengths(ctx, oracle, hccs, Lk):
                                 48, 80, 112, 144, 176, 208, 240, 288, 352, 416, 480, 576, 960, 1152, 2304,
                                 3328, 4608, 7680,
                                 # padded lane groups: the other multiples of 16 up to 4096
-                                272, 304, 336, 528, 544, 1008, 1040, 1104, 2064, 2192, 4080])
+                                272, 304, 336, 528, 544, 1008, 1040, 1104, 2064, 2192, 4080,
+                                4128, 5024, 6144, 8160, 8192])
 @pytest.mark.parametrize("flags", ALL_FLAGS)
 def test_odd_chunk_counts(ctx, oracle, hccs, Lk, flags):
     Lq = 70 if flags & 4 else 37                       # several warps, a ragged last warp, causal rows of every length class
