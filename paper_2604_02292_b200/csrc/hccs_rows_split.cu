@@ -21,7 +21,7 @@
 //
 // Causal rows: masked bytes are replaced by -128 right after the load (they can then never raise
 // the max), their closeness r_m = max(D - m - 128, 0) is subtracted from the sum in closed form,
-// and the output words are masked; the byte masks come from a small shared-memory table.
+// and the output words are masked; the byte masks are computed from the count of valid bytes.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -97,6 +97,13 @@ constexpr uint32_t kSelOdd = 0xB391u;    // bytes 1 and 3, each sign-extended to
 constexpr uint32_t kSelWide = 0x2440u;   // 16-bit pair (r_a, r_b) -> r_a + r_b * 2^24
 constexpr uint32_t kMinus128x4 = 0x80808080u;
 
+// Byte mask of word k of a chunk whose first cnt bytes are valid: 0xff for each valid byte.  Two
+// instructions (add-and-clamp at zero, funnel shift that saturates at 32): a shared-memory table of
+// these masks costs every CTA a fill and a barrier before its first load can be used.
+__device__ __forceinline__ uint32_t byte_mask(int cnt, int k) {
+    return __funnelshift_lc(0xffffffffu, 0u, (uint32_t)__viaddmax_s32(8 * cnt, -32 * k, 0));
+}
+
 // CW: 32-bit words per chunk, 8 (32-byte chunks) or 4 (16-byte chunks, for the row lengths that are a
 // multiple of 16 but not of 32, or whose number of 32-byte chunks has an odd part above 7).
 // PAD: the G*V chunks of a lane group cover more than the row (any multiple of 16 keys: the chunks beyond
@@ -107,14 +114,6 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     constexpr int RW = 32 / G;      // rows per warp
     constexpr int NW = CW * V;      // 32-bit words of logits per lane
     constexpr int CB = 4 * CW;      // bytes (keys) per chunk
-    __shared__ uint32_t mask_tab[CAUSAL ? (CB + 1) * CW : 1];   // [valid bytes of a chunk][word] -> byte mask
-    if (CAUSAL) {
-        for (int idx = threadIdx.x; idx < (CB + 1) * CW; idx += blockDim.x) {
-            const int nb = idx / CW - 4 * (idx % CW);
-            mask_tab[idx] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
-        }
-        __syncthreads();
-    }
     const int lane = threadIdx.x & 31;
     const int sub = lane % G;
     const uint32_t row = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RW + lane / G;
@@ -167,7 +166,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         for (int k = 0; k < CW; ++k) {
             uint32_t w = e[CW * v + k];
             if (CAUSAL) {
-                const uint32_t bm = mask_tab[cnt[v] * CW + k];
+                const uint32_t bm = byte_mask(cnt[v], k);
                 w = (w & bm) | (kMinus128x4 & ~bm);
             }
             const uint32_t ev = prmt(w, 0, kSelEven), od = prmt(w, 0, kSelOdd);
@@ -222,7 +221,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                 const uint32_t pe = e[CW * v + k] * b1 + a1, po = o[CW * v + k] * b1 + a1;
                 uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
                 if (CAUSAL) {
-                    const uint32_t bm = mask_tab[cnt[v] * CW + k];
+                    const uint32_t bm = byte_mask(cnt[v], k);
                     q0 &= prmt(bm, 0, 0x1100u);
                     q1 &= prmt(bm, 0, 0x3322u);
                 }
@@ -273,7 +272,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                     const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
                     q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
                 }
-                if (CAUSAL) q &= mask_tab[cnt[v] * CW + k];
+                if (CAUSAL) q &= byte_mask(cnt[v], k);
                 out[k] = q;
             }
             if constexpr (CW == 8) stg256(p_row + col, out);
