@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (cold L2, so part of the output had not been written back yet); None for workloads
 # that were not captured.  Set back to None when the kernel of a workload changes.
-NCU_TRAFFIC_BYTES = {"config2": 67.13e6 + 15.2e6, "config3": 33.57e6 + 0.7e6, "config4": 201.34e6 + 153.8e6,
+NCU_TRAFFIC_BYTES = {"config2": 67.13e6 + 15.2e6, "config3": 33.57e6 + 0.8e6, "config4": 201.34e6 + 153.8e6,
                      "config5": 75.58e6 + 52.65e6}
 NOMINAL_HBM_GBS = 8000.0
 METRIC = "hccs_forward rows/s (int8 logits -> uint8 probabilities, exact divide)"
