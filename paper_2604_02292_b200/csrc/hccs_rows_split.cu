@@ -14,9 +14,11 @@
 //            every quantity stays non-negative
 //   stage 4  Z = n_valid*F + S*sum(r)       one three-input add per word (16-bit lane sums)
 //   stage 5  rho once per row; p = (F*rho' + S*rho'*r) >> 16 with rho' = rho << (1 - OUT_SHIFT)
-// For uint8 output two elements share one 32x32->64-bit multiply-add: the operand r_a + r_b*2^24
-// times S*rho' plus F*rho'*(1 + 2^24) gives X_a + X_b*2^24 with both X < 2^24 (X = s*rho' <=
-// 255*2^16 because s <= Z), so p_a is byte 2 of the low word and p_b byte 1 of the high word.
+// For uint8 output X = s*rho' < 2^24 (s <= Z), and the two elements of a 16-bit pair are normalised by
+// two 32-bit multiply-adds on the pair: the coefficients are split at 8 bits so that every partial
+// result fits its 16-bit lane (see the kernel).  A 32x32->64-bit multiply-add with the two elements
+// 24 bits apart does the same in one instruction, but its 64-bit addend costs two more on the integer
+// pipe, which is the pipe this kernel is bound by.
 // For uint16 output one 32-bit multiply-add handles a pair directly (s*rho < 2^16).
 //
 // Causal rows: masked bytes are replaced by -128 right after the load (they can then never raise
@@ -86,15 +88,8 @@ __device__ __forceinline__ void stg128(void *p, const uint32_t (&r)[4]) {
                  : "memory");
 }
 
-__device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
-    uint64_t d;
-    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
-    return d;
-}
-
 constexpr uint32_t kSelEven = 0xA280u;   // bytes 0 and 2, each sign-extended to 16 bits
 constexpr uint32_t kSelOdd = 0xB391u;    // bytes 1 and 3, each sign-extended to 16 bits
-constexpr uint32_t kSelWide = 0x2440u;   // 16-bit pair (r_a, r_b) -> r_a + r_b * 2^24
 constexpr uint32_t kMinus128x4 = 0x80808080u;
 
 // Byte mask of word k of a chunk whose first cnt bytes are valid: 0xff for each valid byte.  Two
@@ -108,6 +103,11 @@ __device__ __forceinline__ uint32_t byte_mask(int cnt, int k) {
 // multiple of 16 but not of 32, or whose number of 32-byte chunks has an odd part above 7).
 // PAD: the G*V chunks of a lane group cover more than the row (any multiple of 16 keys: the chunks beyond
 // the row's end are never loaded, count as masked and are not stored); needs the masked instantiation.
+//
+// Masked instantiations decide per chunk index v, once per warp, whether every lane holds a full chunk
+// (then the chunk runs through the unmasked code: no byte masks, no substitution, no output mask), whether
+// no row of the warp reaches it (then it is skipped and stored as zeros), or neither (masked code).  With
+// a causal mask the diagonal crosses exactly one chunk index of a warp, so one chunk per warp pays for masks.
 template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8, bool PAD = false>
 __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, void *p_all, RowArgs a) {
     static_assert(!PAD || CAUSAL, "padded lane groups run through the masked path");
@@ -118,18 +118,21 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     const int sub = lane % G;
     const uint32_t row = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RW + lane / G;
     const bool live = row < (uint32_t)a.rows;
-    uint32_t bidx = 0, head = 0, qi = 0;
-    if (live) row_coords(row, a, bidx, head, qi);
-    int nv = live ? valid_keys_causal<CAUSAL>(qi, a) : 0;
+    // A lane beyond the last row repeats the last row's loads and arithmetic and stores nothing: cheaper
+    // than a fill value for its registers, and every shuffle and vote below stays warp-wide.
+    const uint32_t lrow = min(row, (uint32_t)a.rows - 1u);
+    uint32_t bidx, head, qi;
+    row_coords(lrow, a, bidx, head, qi);
+    int nv = valid_keys_causal<CAUSAL>(qi, a);
     // Programmatic dependent launch: everything above touches no global memory, so it may run
     // while the previous kernel in the stream drains; all reads and writes come after the wait.
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const HeadEntry th = a.table[head];
-    if (CAUSAL && a.key_len && live) nv = min(nv, max(a.key_len[bidx], 0));   // padding mask
+    if (CAUSAL && a.key_len) nv = min(nv, max(a.key_len[bidx], 0));   // padding mask
 
-    // Causal: a chunk index v whose columns lie beyond every row of this warp is skipped
-    // altogether (warp-uniform), e.g. the right half of the first 64 queries of a 128-key head.
+    // Masked: a chunk index v whose columns lie beyond every row of this warp is skipped altogether
+    // (warp-uniform), e.g. the right half of the first 64 queries of a 128-key causal head.
     const int warp_nv = CAUSAL ? __reduce_max_sync(0xffffffffu, nv) : a.Lk;
     auto chunk_used = [&](int v) { return !CAUSAL || v == 0 || v * G * CB < warp_nv; };
     int skipped_cols = 0;           // masked columns of this row that were never materialised
@@ -137,14 +140,16 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     for (int v = 1; v < V; ++v)
         if (!chunk_used(v)) skipped_cols += CB * G;
 
-    // ---- loads: V independent 32-byte requests per lane
+    // ---- loads: V independent requests per lane
     uint32_t e[NW], o[NW];          // first the raw words (in e), then the split lanes
-    int cnt[V];
-    const int8_t *x_row = x_all + (int64_t)row * a.Lk;
+    int cnt[V];                     // valid bytes of this lane's chunk v
+    bool full[V];                   // warp-uniform: every lane's chunk v is complete
+    const int8_t *x_row = x_all + (int64_t)lrow * a.Lk;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int col = (sub + v * G) * CB;
-        cnt[v] = CAUSAL ? min(max(nv - col, 0), CB) : (live ? CB : 0);
+        cnt[v] = CAUSAL ? min(max(nv - col, 0), CB) : CB;
+        full[v] = !CAUSAL || __all_sync(0xffffffffu, cnt[v] == CB);
         uint32_t w[CW];
         if (cnt[v] > 0) {
             if constexpr (CW == 8) ldg256<G == 1>(x_row + col, w);
@@ -162,17 +167,23 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         if (!chunk_used(v)) continue;
+        if (full[v]) {
 #pragma unroll
-        for (int k = 0; k < CW; ++k) {
-            uint32_t w = e[CW * v + k];
-            if (CAUSAL) {
-                const uint32_t bm = byte_mask(cnt[v], k);
-                w = (w & bm) | (kMinus128x4 & ~bm);
+            for (int k = CW * v; k < CW * v + CW; ++k) {
+                const uint32_t w = e[k];
+                e[k] = prmt(w, 0, kSelEven);
+                o[k] = prmt(w, 0, kSelOdd);
+                M = __vimax3_s16x2(M, e[k], o[k]);
             }
-            const uint32_t ev = prmt(w, 0, kSelEven), od = prmt(w, 0, kSelOdd);
-            e[CW * v + k] = ev;
-            o[CW * v + k] = od;
-            M = __vimax3_s16x2(M, ev, od);
+        } else {
+#pragma unroll
+            for (int k = 0; k < CW; ++k) {
+                const uint32_t bm = byte_mask(cnt[v], k);
+                const uint32_t w = (e[CW * v + k] & bm) | (kMinus128x4 & ~bm);
+                e[CW * v + k] = prmt(w, 0, kSelEven);
+                o[CW * v + k] = prmt(w, 0, kSelOdd);
+                M = __vimax3_s16x2(M, e[CW * v + k], o[CW * v + k]);
+            }
         }
     }
     int m = max((int)(short)(M & 0xffffu), (int)M >> 16);
@@ -215,18 +226,21 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
             if (!chunk_used(v)) {
 #pragma unroll
                 for (int k = 0; k < 2 * CW; ++k) out[k] = 0;
-            } else
+            } else {
 #pragma unroll
-            for (int k = 0; k < CW; ++k) {
-                const uint32_t pe = e[CW * v + k] * b1 + a1, po = o[CW * v + k] * b1 + a1;
-                uint32_t q0 = prmt(pe, po, 0x5410u), q1 = prmt(pe, po, 0x7632u);
-                if (CAUSAL) {
-                    const uint32_t bm = byte_mask(cnt[v], k);
-                    q0 &= prmt(bm, 0, 0x1100u);
-                    q1 &= prmt(bm, 0, 0x3322u);
+                for (int k = 0; k < CW; ++k) {
+                    const uint32_t pe = e[CW * v + k] * b1 + a1, po = o[CW * v + k] * b1 + a1;
+                    out[2 * k] = prmt(pe, po, 0x5410u);
+                    out[2 * k + 1] = prmt(pe, po, 0x7632u);
                 }
-                out[2 * k] = q0;
-                out[2 * k + 1] = q1;
+                if (!full[v]) {
+#pragma unroll
+                    for (int k = 0; k < CW; ++k) {
+                        const uint32_t bm = byte_mask(cnt[v], k);
+                        out[2 * k] &= prmt(bm, 0, 0x1100u);
+                        out[2 * k + 1] &= prmt(bm, 0, 0x3322u);
+                    }
+                }
             }
             if constexpr (CW == 8) {
                 uint32_t lo[8], hi[8];
@@ -242,6 +256,12 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         const int sh = 1 - a.out_shift;                    // 0 or 1 (checked by the launcher)
         const uint32_t rp = rho << sh;
         const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
+        // Exact divide: X = a1 + b1*r = s*rho' < 2^24 (s <= Z), p = X >> 16.  With a1 = ah*256 + al and
+        // b1 = bh*256 + bl, X >> 8 = ah + bh*r + ((al + bl*r) >> 8) =: Y < 2^16, and both ah + bh*r and
+        // al + bl*r (r <= 127) fit 16 bits: a pair of elements takes two 32-bit multiply-adds on its 16-bit
+        // lanes, one byte permute for the carry, one add, and p is the high byte of each lane of Y.
+        const uint32_t ah2 = (a1 >> 8) * 0x00010001u, al2 = (a1 & 255u) * 0x00010001u;
+        const uint32_t bh = b1 >> 8, bl = b1 & 255u;
         uint8_t *p_row = (uint8_t *)p_all + (int64_t)row * a.Lk;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
@@ -251,29 +271,27 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
             if (!chunk_used(v)) {
 #pragma unroll
                 for (int k = 0; k < CW; ++k) out[k] = 0;
-            } else
+            } else {
 #pragma unroll
-            for (int k = 0; k < CW; ++k) {
-                uint32_t q;
-                if (!CLB) {
-                    const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
-                    const uint64_t pe = mad_wide(prmt(e[CW * v + k], 0, kSelWide), b1, A);
-                    const uint64_t po = mad_wide(prmt(o[CW * v + k], 0, kSelWide), b1, A);
-                    // bytes 2,3 of the high words are zero: [p0,0,p2,0] + [0,p1,0,p3]
-                    const uint32_t t0 = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u);
-                    const uint32_t t1 = prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
-                    q = t0 + t1;
-                } else {
-                    // the leading-bit reciprocal can overshoot 255: saturate each element
-                    const uint32_t ev = e[CW * v + k], od = o[CW * v + k];
-                    const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
-                    const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
-                    const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
-                    const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
-                    q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                for (int k = 0; k < CW; ++k) {
+                    const uint32_t re = e[CW * v + k], ro = o[CW * v + k];
+                    if (!CLB) {
+                        const uint32_t ye = re * bh + ah2 + prmt(re * bl + al2, 0, 0x4341u);
+                        const uint32_t yo = ro * bh + ah2 + prmt(ro * bl + al2, 0, 0x4341u);
+                        out[k] = prmt(ye, yo, 0x7351u);
+                    } else {
+                        // the leading-bit reciprocal can overshoot 255: saturate each element
+                        const uint32_t x0 = min(a1 + b1 * (re & 0xffffu), 0x00ffffffu);
+                        const uint32_t x1 = min(a1 + b1 * (ro & 0xffffu), 0x00ffffffu);
+                        const uint32_t x2 = min(a1 + b1 * (re >> 16), 0x00ffffffu);
+                        const uint32_t x3 = min(a1 + b1 * (ro >> 16), 0x00ffffffu);
+                        out[k] = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                    }
                 }
-                if (CAUSAL) q &= byte_mask(cnt[v], k);
-                out[k] = q;
+                if (!full[v]) {
+#pragma unroll
+                    for (int k = 0; k < CW; ++k) out[k] &= byte_mask(cnt[v], k);
+                }
             }
             if constexpr (CW == 8) stg256(p_row + col, out);
             else stg128(p_row + col, out);
