@@ -23,8 +23,15 @@
  *     the default stream) and the call returns without synchronising, unless
  *     stated otherwise.
  *   - Errors are return codes only.  On any error nothing is launched.
- *   - A context is not thread-safe: one call at a time per context (different contexts, also on
- *     the same device, are independent).
+ *   - A context is not thread-safe: one host call at a time per context (different contexts, also
+ *     on the same device, are independent).  On the GPU, hccs_forward, hccs_forward_keylen and
+ *     hccs_forward_host calls of one context only read the context's parameter table and may
+ *     overlap each other freely (different streams, back to back on one stream).  Calls that rewrite
+ *     device memory the context owns do so on their own `cuda_stream`: hccs_params_upload (the
+ *     parameter table) and the hccs_attention_fused* calls (a small per-head multiplier table,
+ *     rewritten only when the multipliers, the shift or the output scales differ from the previous
+ *     fused call's).  Order such a call against other work of the same context that may still be
+ *     running on another stream yourself (an event, or one stream per context).
  *   - There is no CPU implementation behind this interface.
  */
 #ifndef HCCS_H
@@ -79,9 +86,11 @@ hccs_status_t hccs_destroy(hccs_ctx_t *ctx);
  *   out_shift  OUT_SHIFT of the int8 output path (Eq. 8), 0..8; 0 unless you know better
  *   bad_head   may be NULL; receives the first offending head on HCCS_ERR_CONSTRAINT, else -1
  * Every item of the paper's Section "Integer Range Constraints" is checked on the host for
- * n = n_design:  1 <= Dmax <= 127;  S >= 0;  B - S*Dmax >= ceil(256/n);  n*B <= 32767 (hence
- * B <= 32767); and S <= 127 (S is an operand of a single int8 multiply-accumulate).  On a
- * violation nothing is uploaded and the previous table stays in force.
+ * n = n_design:  Dmax <= 127;  S >= 0;  B - S*Dmax >= ceil(256/n);  n*B <= 32767 (hence
+ * B <= 32767).  Two more bounds are this library's own additions, not the paper's: Dmax >= 1 (a
+ * clamp bound of 0 would make every row uniform) and S <= 127 (the paper describes the score as a
+ * single int8 multiply-accumulate, so S is kept an int8 operand).  On a violation nothing is
+ * uploaded and the previous table stays in force.
  * The table is copied from an internal pinned staging buffer on `cuda_stream`; `params` may be
  * reused as soon as the call returns.  The first upload (or one with more heads than before)
  * allocates device memory and therefore synchronises the device.
@@ -217,6 +226,21 @@ hccs_status_t hccs_calibrate(const int8_t *logits, int32_t B, int32_t H, int32_t
  * receives it. */
 hccs_status_t hccs_device_status(hccs_ctx_t *ctx, uint32_t *word, void *cuda_stream);
 
+/*
+ * Self-test of the device-side wait limits.  (The paper has no counterpart.)  Every wait of the
+ * TMA-staged kernels (on a bulk copy, on a tensor-core commit) gives up after a limit of SM clock
+ * cycles -- about a second in production -- sets a bit of the status word and lets the kernel return
+ * instead of hanging the GPU.  This call runs that give-up path on purpose and harmlessly: one small
+ * CTA waits, through the same wait routines, on a barrier that nothing will ever complete, with the
+ * limit given here.
+ *   mode          0: the wait of the long-row kernel (sets bit 0 of the status word);
+ *                 1: the abort-flag wait of the fused kernel (sets bit 1; a second thread gives up
+ *                    because it sees the flag, not because its own, longer limit ran out)
+ *   limit_cycles  1 .. 10 000 000
+ * Afterwards hccs_device_status returns HCCS_ERR_DEVICE_TIMEOUT once and clears the word.
+ */
+hccs_status_t hccs_debug_wait_timeout(hccs_ctx_t *ctx, int32_t mode, int64_t limit_cycles, void *cuda_stream);
+
 /* The cudaError_t of the last failing CUDA call made through this context (0 = none). */
 int32_t hccs_last_cuda_error(const hccs_ctx_t *ctx);
 
@@ -237,21 +261,25 @@ uint64_t hccs_launch_count(const hccs_ctx_t *ctx);
  * cannot create an hccs_ctx_t, because the context allocates its parameter table.
  *
  * What it does: the same result as hccs_forward, computed by the shared-memory-staged
- * one-CTA-per-row kernel, with all of the library's working memory (parameter table, the row
- * counter of the persistent CTAs, the status word) in one fixed 4.25 KB array that is part of
- * the loaded library image on every GPU.  No context, no cudaMalloc/cudaFree, no allocating
- * library call; the tensors are the caller's.
+ * one-CTA-per-row kernel, with all of the library's working memory (the parameter table and the
+ * status word that device-side waits report to) in one fixed 4.25 KB array that is part of the
+ * loaded library image on every GPU.  No context, no cudaMalloc/cudaFree, no allocating library
+ * call, no host-to-device copy; the tensors are the caller's.
  *   params, num_heads, n_design, out_shift   HOST table, checked exactly as hccs_params_upload
- *        does; num_heads above 256 does not fit the fixed array: HCCS_ERR_UNSUPPORTED
+ *        does; it travels to the GPU as a kernel argument, so it may be reused or freed as soon as
+ *        the call returns.  num_heads above 256 does not fit the fixed array: HCCS_ERR_UNSUPPORTED
  *   logits, probs, B, H, Lq, Lk, flags       as hccs_forward, on the CURRENT device; this entry
  *        point needs Lk % 16 == 0 and 16-byte aligned pointers (else HCCS_ERR_UNSUPPORTED)
- *   timed_out   NULL: fully asynchronous.  Non-NULL (host): the call synchronises `cuda_stream`
- *        and stores the status word there; non-zero also returns HCCS_ERR_DEVICE_TIMEOUT.
- * The first call on each device looks up the device address of the fixed array; make that
- * first call outside any stream capture.  All calls on a device share the array and it keeps
- * the previous call's contents: each call rewrites the table and clears the counter and status
- * on `cuda_stream` before its kernel.  Two calls whose work overlaps on the GPU (different
- * streams, no dependency between them) therefore race on it -- serialise them.
+ *   timed_out   NULL: two kernels are enqueued on `cuda_stream` (one that fills the array, then the
+ *        row kernel) and the call returns without waiting for them.  Non-NULL (host): the call
+ *        also synchronises `cuda_stream` and stores the status word there; non-zero returns
+ *        HCCS_ERR_DEVICE_TIMEOUT as well.
+ * The first call on each device looks up the device address of the fixed array
+ * (cudaGetSymbolAddress); make that first call before any stream capture begins.  All calls on a
+ * device share the array and it keeps the previous call's contents: each call rewrites the table
+ * and clears the status word on `cuda_stream` before its row kernel.  Two calls whose work
+ * overlaps on the GPU (different streams, no dependency between them) therefore race on it --
+ * serialise them.
  */
 hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *params, int32_t num_heads,
                                           int32_t n_design, int32_t out_shift,

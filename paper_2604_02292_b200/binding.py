@@ -38,7 +38,7 @@ HCCS_CAUSAL = 4
 EXPORTS = ("hccs_create", "hccs_destroy", "hccs_params_check", "hccs_params_upload", "hccs_forward",
            "hccs_forward_keylen", "hccs_forward_host",
            "hccs_attention_fused", "hccs_attention_fused_keylen", "hccs_attention_fused_f32", "hccs_device_status", "hccs_last_cuda_error", "hccs_status_string",
-           "hccs_launch_count", "hccs_forward_static_scratch", "hccs_calibrate")
+           "hccs_launch_count", "hccs_forward_static_scratch", "hccs_calibrate", "hccs_debug_wait_timeout")
 
 _vp, _i32, _u32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32
 
@@ -73,6 +73,8 @@ _lib.hccs_status_string.argtypes = [ctypes.c_int]
 _lib.hccs_status_string.restype = ctypes.c_char_p
 _lib.hccs_launch_count.argtypes = [_vp]
 _lib.hccs_launch_count.restype = ctypes.c_uint64
+_lib.hccs_debug_wait_timeout.argtypes = [_vp, _i32, ctypes.c_int64, _vp]
+_lib.hccs_debug_wait_timeout.restype = ctypes.c_int
 
 
 _lib.hccs_forward_static_scratch.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _i32, _u32,
@@ -257,6 +259,12 @@ class Context:
         if st not in (HCCS_OK, HCCS_ERR_DEVICE_TIMEOUT):
             raise HccsError(st, "hccs_device_status")
         return int(w.value)
+
+    # -- hccs_debug_wait_timeout
+    def hccs_debug_wait_timeout(self, mode: int, limit_cycles: int, stream=None) -> None:
+        st = _lib.hccs_debug_wait_timeout(self._h, int(mode), int(limit_cycles), _stream_ptr(stream))
+        if st != HCCS_OK:
+            raise HccsError(st, "hccs_debug_wait_timeout")
 
     def hccs_last_cuda_error(self) -> int:
         return int(_lib.hccs_last_cuda_error(self._h))

@@ -14,11 +14,13 @@ struct hccs_ctx {
     hccs::HeadEntry *h_table = nullptr;     // pinned staging copy of it
     int32_t *d_mult = nullptr;              // device copy of the fused path's per-head multipliers
     int32_t *h_mult = nullptr;              // pinned staging for them
+    int32_t *mult_last = nullptr;           // host copy of what d_mult holds (to skip an unchanged upload)
+    int32_t mult_last_heads = 0;            // 0: d_mult holds nothing yet
     int32_t capacity = 0;                   // heads the allocations can hold
     int32_t num_heads = 0;                  // 0 = nothing uploaded
     int32_t n_design = 0;
     int32_t out_shift = 0;
-    uint32_t *d_status = nullptr;           // device scratch: word 0 status, word 1 row counter
+    uint32_t *d_status = nullptr;           // device status word (bounded waits report here)
     uint32_t *h_status = nullptr;           // pinned landing place for it
     cudaEvent_t table_copied = nullptr;     // the staging buffers may be rewritten after this
     cudaEvent_t mult_copied = nullptr;
@@ -98,13 +100,17 @@ hccs_status_t ensure_capacity(hccs_ctx *ctx, int32_t heads) {
     if (ctx->h_table) cudaFreeHost(ctx->h_table);
     if (ctx->d_mult) cudaFree(ctx->d_mult);
     if (ctx->h_mult) cudaFreeHost(ctx->h_mult);
+    delete[] ctx->mult_last;
     ctx->d_table = nullptr; ctx->h_table = nullptr; ctx->d_mult = nullptr; ctx->h_mult = nullptr;
+    ctx->mult_last = nullptr; ctx->mult_last_heads = 0;
     ctx->capacity = 0;
     int32_t cap = heads < 64 ? 64 : heads;
     HCCS_CUDA(ctx, cudaMalloc(&ctx->d_table, sizeof(hccs::HeadEntry) * cap));
     HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_table, sizeof(hccs::HeadEntry) * cap, cudaHostAllocDefault));
     HCCS_CUDA(ctx, cudaMalloc(&ctx->d_mult, sizeof(int32_t) * 8 * cap));
     HCCS_CUDA(ctx, cudaHostAlloc(&ctx->h_mult, sizeof(int32_t) * 8 * cap, cudaHostAllocDefault));
+    ctx->mult_last = new (std::nothrow) int32_t[8 * (size_t)cap];
+    if (!ctx->mult_last) return HCCS_ERR_CUDA;
     ctx->capacity = cap;
     return HCCS_OK;
 }
@@ -128,7 +134,7 @@ hccs::RowArgs make_row_args(const hccs_ctx *ctx, int32_t rows, int32_t H, int32_
     hccs::RowArgs a;
     a.table = ctx->d_table;
     a.status = ctx->d_status;
-    a.row_counter = ctx->d_status + 1;
+    a.wait_cycles = hccs::kDefaultWaitCycles;
     a.rows = rows;
     a.H = H;
     a.Lq = Lq;
@@ -187,6 +193,7 @@ hccs_status_t hccs_destroy(hccs_ctx_t *ctx) {
     if (ctx->h_table) cudaFreeHost(ctx->h_table);
     if (ctx->d_mult) cudaFree(ctx->d_mult);
     if (ctx->h_mult) cudaFreeHost(ctx->h_mult);
+    delete[] ctx->mult_last;
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     if (ctx->table_copied) cudaEventDestroy(ctx->table_copied);
@@ -360,13 +367,19 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     DeviceGuard g(ctx->device);
     if (!g.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    HCCS_CUDA(ctx, cudaEventSynchronize(ctx->mult_copied));
     // Per head: {multiplier, and for shifts up to 24 the constants of the single-multiply
     // requantisation: multiplier << k, offset, -lo, hi - lo} (see hccs_fused.cu, phase 1), then the
     // fp32 output scale, a spare word and 1 / multiplier as a double; eight 32-bit words per head.
+    // The words are built on the stack and go up only when they differ from what the device table
+    // already holds (the usual case is the same multipliers call after call): then nothing is copied
+    // and the host never waits for an earlier call's copy.
+    constexpr int32_t kStackHeads = 64;
+    int32_t stack_words[8 * kStackHeads];
+    int32_t *words = H <= kStackHeads ? stack_words : new (std::nothrow) int32_t[8 * (size_t)H];
+    if (!words) return HCCS_ERR_INVALID_ARG;
     for (int32_t h = 0; h < H; ++h) {
         const int64_t M = requant_mult[h];
-        int32_t *e = ctx->h_mult + 8 * h;
+        int32_t *e = words + 8 * h;
         e[0] = (int32_t)M;
         e[1] = e[2] = e[3] = e[5] = e[6] = e[7] = 0;
         const float scale = out_scale ? out_scale[h] : 1.0f;
@@ -389,14 +402,34 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
             e[3] = (int32_t)(hi - lo);
         }
     }
-    HCCS_CUDA(ctx, cudaMemcpyAsync(ctx->d_mult, ctx->h_mult, sizeof(int32_t) * 8 * H,
-                                   cudaMemcpyHostToDevice, stream));
-    HCCS_CUDA(ctx, cudaEventRecord(ctx->mult_copied, stream));
+    const bool same = ctx->mult_last_heads == H && memcmp(ctx->mult_last, words, sizeof(int32_t) * 8 * H) == 0;
+    if (!same) {
+        // the pinned staging copy may still be in flight from the previous upload
+        cudaError_t e = cudaEventSynchronize(ctx->mult_copied);
+        if (e == cudaSuccess) {
+            memcpy(ctx->h_mult, words, sizeof(int32_t) * 8 * H);
+            e = cudaMemcpyAsync(ctx->d_mult, ctx->h_mult, sizeof(int32_t) * 8 * H, cudaMemcpyHostToDevice, stream);
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->mult_copied, stream);
+        if (e == cudaSuccess) {
+            memcpy(ctx->mult_last, words, sizeof(int32_t) * 8 * H);
+            ctx->mult_last_heads = H;
+        } else {
+            ctx->mult_last_heads = 0;
+        }
+        if (words != stack_words) delete[] words;
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    } else {
+        if (words != stack_words) delete[] words;
+        // the table went up on the stream of an earlier call: order this stream behind that copy
+        HCCS_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->mult_copied, 0));
+    }
     hccs::FusedArgs a;
     a.Q = Q; a.K = K; a.V = V; a.O = O;
     a.table = ctx->d_table;
     a.requant_mult = ctx->d_mult;
     a.status = ctx->d_status;
+    a.wait_cycles = hccs::kDefaultWaitCycles;
     a.out_f32 = out_scale ? 1 : 0;
     a.key_len = key_len;
     a.requant_shift = requant_shift;
@@ -444,6 +477,16 @@ hccs_status_t hccs_device_status(hccs_ctx_t *ctx, uint32_t *word, void *cuda_str
     const uint32_t w = *ctx->h_status;
     if (word) *word = w;
     return w ? HCCS_ERR_DEVICE_TIMEOUT : HCCS_OK;
+}
+
+hccs_status_t hccs_debug_wait_timeout(hccs_ctx_t *ctx, int32_t mode, int64_t limit_cycles, void *cuda_stream) {
+    if (!ctx || (mode != 0 && mode != 1)) return HCCS_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > 10000000) return HCCS_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+    HCCS_CUDA(ctx, hccs::launch_wait_probe(ctx->d_status, mode, (long long)limit_cycles, (cudaStream_t)cuda_stream));
+    ctx->launches += 1;
+    return HCCS_OK;
 }
 
 int32_t hccs_last_cuda_error(const hccs_ctx_t *ctx) { return ctx ? ctx->last_cuda_error : 0; }

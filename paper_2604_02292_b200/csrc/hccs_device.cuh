@@ -60,4 +60,45 @@ __device__ __forceinline__ int valid_keys(uint32_t b, uint32_t i, const RowArgs 
     return nv;
 }
 
+// ---- mbarrier waits with a limit (shared by the TMA-staged row kernel, the fused kernel and the
+// wait-limit probe): no wait in this library spins without one.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+// Waits for the phase with the given parity for at most `limit_cycles` SM clock cycles; false when the
+// limit ran out (the caller records it in the status word and leaves).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit_cycles) {
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+}
+// The same for a CTA whose threads wait on many barriers: the first wait that runs out raises the CTA's
+// abort flag and sets `status_bit` in the status word; every other wait sees the flag and gives up too.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                    uint32_t *status, uint32_t status_bit, long long limit_cycles) {
+    long long t0 = 0;
+    for (uint32_t polls = 0;; ++polls) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((polls & 31u) != 31u) continue;          // look at the flag and the clock now and then
+        if (*abort_flag) return false;
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        if (now - t0 > limit_cycles) {
+            *abort_flag = 1;
+            atomicOr(status, status_bit);
+            return false;
+        }
+    }
+}
+
 }  // namespace hccs

@@ -54,7 +54,6 @@ constexpr uint32_t kTmemCols = 512;       // S0 [0,128)  S1 [128,256)  S2 [256,3
 constexpr int kSBufs = 3;                 // S blocks in flight between the tensor core and the row warps
 constexpr uint32_t kTmemO = 384;
 constexpr uint32_t kOBoxBytes = 128 * 128; // one staged box of the output tile: 128 rows x 32 int32 columns
-constexpr long long kWaitCycles = 2000000000ll;
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -96,28 +95,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 // Bounded, abort-aware wait.  Returns false when the wait was given up (here or elsewhere).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          uint32_t *status) {
-    long long t0 = 0;
-    for (uint32_t polls = 0;; ++polls) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if ((polls & 31u) != 31u) continue;          // look at the flag and the clock now and then
-        if (*abort_flag) return false;
-        const long long now = clock64();
-        if (t0 == 0) t0 = now;
-        if (now - t0 > kWaitCycles) {
-            *abort_flag = 1;
-            atomicOr(status, STATUS_FUSED_TIMEOUT);
-            return false;
-        }
-    }
+                                          uint32_t *status, long long limit_cycles) {
+    return mbar_wait_abortable(bar, parity, abort_flag, status, STATUS_FUSED_TIMEOUT, limit_cycles);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -295,14 +274,14 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 const int bh = tile / nblk;
                 const int kblocks = blocks_of(tile);
                 // the other K blocks land where the previous tile's V sits: wait for its last MMA
-                if (it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (it - 1) & 1, abortp, a.status);
+                if (it > 0) ok = mbar_wait(smem_u32(&bars.o_full), (it - 1) & 1, abortp, a.status, a.wait_cycles);
                 if (!ok) break;
                 for (int kb = 2 + me; kb < kblocks; kb += 2) {
                     load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
                 // V takes the K buffer once the first contraction has read the last K block; Q and
                 // the first K blocks of the next tile are fetched as well
-                ok = mbar_wait(smem_u32(&bars.k_done), it & 1, abortp, a.status);
+                ok = mbar_wait(smem_u32(&bars.k_done), it & 1, abortp, a.status, a.wait_cycles);
                 if (!ok) break;
                 // (the next tile's Q and K go after the first V block, early enough for its first round
                 // to start behind the probability pass)
@@ -329,7 +308,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const uint32_t dk_lo = (uint32_t)dk, dk_hi = (uint32_t)(dk >> 32);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int kblocks = blocks_of(tile);
-                ok = mbar_wait(smem_u32(&bars.q_full), it & 1, abortp, a.status);
+                ok = mbar_wait(smem_u32(&bars.q_full), it & 1, abortp, a.status, a.wait_cycles);
                 // the scan flow of the row warps reads every S block twice: once for the row maximum,
                 // once to requantise
                 for (int round = 0; ok && round < (two_rounds ? 2 : 1); ++round) {
@@ -341,10 +320,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         ++g;
                         if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
                         if (!mine) continue;
-                        if (cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (cyc - 1) & 1, abortp, a.status);
+                        if (cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (cyc - 1) & 1, abortp, a.status, a.wait_cycles);
                         // the K block's copy must have landed: in the second round too, where the
                         // block may fall to the issuer that did not wait for it in the first
-                        if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status);
+                        if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status, a.wait_cycles);
                         if (!ok) break;
                         tcgen05_fence_after();
                         // K block kb sits (kb < 2 ? kb : kb + 2) tiles above the first prefetch slot;
@@ -381,8 +360,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                 for (int kb = 0; kb < kMaxBlocks; ++kb) {
                     if (kb >= kblocks) break;
-                    ok = mbar_wait(smem_u32(&bars.v_full[kb]), (p_par >> kb) & 1, abortp, a.status);
-                    if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[kb]), (p_par >> kb) & 1, abortp, a.status);
+                    ok = mbar_wait(smem_u32(&bars.v_full[kb]), (p_par >> kb) & 1, abortp, a.status, a.wait_cycles);
+                    if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[kb]), (p_par >> kb) & 1, abortp, a.status, a.wait_cycles);
                     if (!ok) break;
                     p_par ^= 1u << kb;
                     tcgen05_fence_after();
@@ -413,7 +392,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         // one S block of the first round: the running maximum of the row's raw accumulators
         auto first_round_block = [&](int kb, int nv_row, int &amax) {
             const uint32_t sb = s_buf;
-            ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
+            ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status, a.wait_cycles);
             if (!ok) return;
             if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
             tcgen05_fence_after();
@@ -515,7 +494,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     ((uint32_t)((int64_t)lo_t * M + R) << kk) - ((uint32_t)(-cm) << 24);
                 for (int kb = 0; ok && kb < kblocks; ++kb) {
                     const uint32_t sb = s_buf;
-                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status, a.wait_cycles);
                     if (!ok) break;
                     if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
                     tcgen05_fence_after();
@@ -543,7 +522,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 const int32_t mult_hi = rq.x << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
                 for (int kb = 0; ok && kb < kblocks; ++kb) {
                     const uint32_t sb = s_buf;
-                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status);
+                    ok = mbar_wait(smem_u32(&bars.s_full[sb]), s_cyc & 1, abortp, a.status, a.wait_cycles);
                     if (!ok) break;
                     if (++s_buf == kSBufs) { s_buf = 0; ++s_cyc; }
                     tcgen05_fence_after();
@@ -664,7 +643,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // layout -- which also spreads a warp's 16-byte stores over all banks -- and one thread
             // sends both boxes off as tiled bulk stores; rows beyond L fall outside the tensor map
             // and are dropped.
-            if (ok) ok = mbar_wait(smem_u32(&bars.o_full), it & 1, abortp, a.status);
+            if (ok) ok = mbar_wait(smem_u32(&bars.o_full), it & 1, abortp, a.status, a.wait_cycles);
             if (ok) {
                 tcgen05_fence_after();
                 constexpr int kCols = D / 4;                      // columns of O per thread: 16 or 32

@@ -27,7 +27,7 @@ FastDiv make_fastdiv(uint32_t d);
 struct RowArgs {
     const HeadEntry *table;   // device, num_heads entries
     uint32_t *status;         // device status word (bounded waits report here)
-    uint32_t *row_counter;    // device scratch word: next row of the CTA-per-row kernel (zeroed per launch)
+    long long wait_cycles;    // limit of every device-side wait, in SM clock cycles
     int32_t rows;             // B*H*Lq
     int32_t H, Lq, Lk;
     int32_t causal_off;       // Lk - Lq
@@ -52,6 +52,7 @@ struct FusedArgs {
     int32_t out_f32;               // 1: O = float(acc) * scale_h
     const int32_t *key_len;        // device, one entry per batch entry, or NULL: keys beyond key_len[b] are padding
     uint32_t *status;
+    long long wait_cycles;         // limit of every device-side wait, in SM clock cycles
     int32_t requant_shift;
     int32_t B, H, L, d;
     int32_t out_shift;
@@ -72,5 +73,10 @@ cudaError_t try_launch_cta(const int8_t *logits, void *probs, const RowArgs &a, 
                            cudaStream_t stream, bool *taken);
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches);
 bool fused_shape_supported(int32_t L, int32_t d);
+// One CTA that waits on an mbarrier nobody arrives on, through the production wait helpers, with the given
+// limit: mode 0 the plain bounded wait (STATUS_ROW_TMA_TIMEOUT), mode 1 the abortable one (STATUS_FUSED_TIMEOUT).
+cudaError_t launch_wait_probe(uint32_t *status, int mode, long long limit_cycles, cudaStream_t stream);
+
+constexpr long long kDefaultWaitCycles = 2000000000ll;   // about one second of SM clocks
 
 }  // namespace hccs

@@ -1,15 +1,16 @@
 // CTA-per-row kernel for long rows (Lk % 16 == 0, up to 32752 keys): Algorithm 1 with the row
 // staged in shared memory.
 //
-// Persistent CTAs take rows from a global counter (rows cost different amounts of work under a
-// causal mask).  For every row one thread issues a 1-D bulk asynchronous copy (TMA,
+// Persistent CTAs walk over the rows with a stride of the grid size (neighbouring rows go to different
+// CTAs, which also spreads the cheap and the costly rows of a causal mask; no counter, no scratch word
+// that two launches could share).  For every row one thread issues a 1-D bulk asynchronous copy (TMA,
 // cp.async.bulk) of the row's valid prefix into one of two shared-memory stages; the copy of
 // the next row is in flight while the CTA makes its three passes over the current one:
 //   pass 1  row max (Eq. 1)            pass 2  sum of the clamped scores (Eq. 2, 3, 5)
 //   once    reciprocal (Eq. 6 / 8 / 9) pass 3  normalise (Eq. 7 / int8 output path) into an
 //                                              output stage, written back by a bulk store.
 // The element arithmetic is the same 16-bit-pair formulation as the register-resident kernel.
-// Every wait on an mbarrier is bounded: when it runs out the CTA records
+// Every wait on an mbarrier is bounded (RowArgs::wait_cycles): when it runs out the CTA records
 // STATUS_ROW_TMA_TIMEOUT in the status word and stops taking rows.  No multicast, no clusters.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -24,7 +25,6 @@ namespace hccs {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr long long kWaitCycles = 2000000000ll;   // about one second of SM clocks: then a wait is given up
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -34,32 +34,11 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
-__device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
-    uint64_t d;
-    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
-    return d;
-}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    const long long t0 = clock64();
-    for (;;) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if (clock64() - t0 > kWaitCycles) return false;
-    }
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile(
@@ -119,10 +98,12 @@ __global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all,
     const int tid = threadIdx.x;
     const uint32_t bar[2] = {smem_u32(&full_bar[0]), smem_u32(&full_bar[1])};
 
-    // thread 0: take the next row from the counter and start its copy into stage s
+    // thread 0: this CTA's next row (stride = grid size); start its copy into stage s
+    int64_t next_row = blockIdx.x;
     auto fetch = [&](int s) {
         RowJob j;
-        j.row = (int32_t)atomicAdd(a.row_counter, 1u);
+        j.row = (int32_t)min(next_row, (int64_t)a.rows);
+        next_row += gridDim.x;
         j.nv = 0; j.head = 0; j.bytes = 0;
         if (j.row >= a.rows) {
             j.row = -1;
@@ -158,14 +139,17 @@ __global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all,
         if (j.row < 0) break;
         bool ok = true;
         if (j.bytes) {
-            ok = mbar_wait(bar[s], phase[s]);
+            ok = mbar_wait_bounded(bar[s], phase[s], a.wait_cycles);
             phase[s] ^= 1;
         }
         if (!__syncthreads_and(ok)) {                 // uniform decision: give up together
             if (tid == 0) {
                 atomicOr(a.status, STATUS_ROW_TMA_TIMEOUT);
-                // give the copy that was started for the other stage a bounded chance to land
-                if (job[s ^ 1].row >= 0 && job[s ^ 1].bytes) (void)mbar_wait(bar[s ^ 1], phase[s ^ 1]);
+                // shared memory must outlive the copies in flight: this stage's and the one started for
+                // the other stage get the full default limit to land, whatever limit the wait above had
+                (void)mbar_wait_bounded(bar[s], phase[s] ^ 1, kDefaultWaitCycles);
+                if (job[s ^ 1].row >= 0 && job[s ^ 1].bytes)
+                    (void)mbar_wait_bounded(bar[s ^ 1], phase[s ^ 1], kDefaultWaitCycles);
             }
             break;
         }
@@ -245,9 +229,12 @@ __global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all,
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
             }
         } else if (a.out_shift <= 1) {
-            const uint32_t rp = rho << (1 - a.out_shift);
+            // the same pair arithmetic as the register-resident kernel: X = s * rho' < 2^24, coefficients split
+            // at 8 bits so that every partial result fits a 16-bit lane
+            const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
             const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
-            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+            const uint32_t ah2 = (a1 >> 8) * 0x00010001u, al2 = (a1 & 255u) * 0x00010001u;
+            const uint32_t bh = b1 >> 8, bl = b1 & 255u;
             for (int v = tid; v < total_vec; v += kThreads) {
                 uint32_t o[4] = {0, 0, 0, 0};
                 if (v < nvec) {
@@ -259,16 +246,13 @@ __global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all,
                         const uint32_t od = __viaddmax_s16x2(prmt(w[k], 0, 0xB391u), c2, 0u);
                         uint32_t q;
                         if (!CLB) {
-                            const uint64_t pe = mad_wide(prmt(ev, 0, 0x2440u), b1, A);
-                            const uint64_t po = mad_wide(prmt(od, 0, 0x2440u), b1, A);
-                            q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) +
-                                prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                            const uint32_t ye = ev * bh + ah2 + prmt(ev * bl + al2, 0, 0x4341u);
+                            const uint32_t yo = od * bh + ah2 + prmt(od * bl + al2, 0, 0x4341u);
+                            q = prmt(ye, yo, 0x7351u);
                         } else {
-                            const uint32_t x0 = min(a1 + b1 * (ev & 0xffffu), 0x00ffffffu);
-                            const uint32_t x1 = min(a1 + b1 * (od & 0xffffu), 0x00ffffffu);
-                            const uint32_t x2 = min(a1 + b1 * (ev >> 16), 0x00ffffffu);
-                            const uint32_t x3 = min(a1 + b1 * (od >> 16), 0x00ffffffu);
-                            q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                            const uint32_t ye = __viaddmin_u16x2(ev * bh + ah2, prmt(ev * bl + al2, 0, 0x4341u), 0x7fff7fffu);
+                            const uint32_t yo = __viaddmin_u16x2(od * bh + ah2, prmt(od * bl + al2, 0, 0x4341u), 0x7fff7fffu);
+                            q = prmt(ye >> 7, yo >> 7, 0x6240u);
                         }
                         if (CAUSAL) q &= byte_prefix_mask(j.nv - 16 * v - 4 * k);
                         o[k] = q;
@@ -317,8 +301,6 @@ cudaError_t launch_cta(const int8_t *x, void *p, const RowArgs &a, cudaStream_t 
     auto kernel = rows_cta_kernel<U16, CLB, CAUSAL>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(a.row_counter, 0, sizeof(uint32_t), st);
-    if (e != cudaSuccess) return e;
     int ctas_per_sm = (int)((200u * 1024u) / (smem + 1024));
     if (ctas_per_sm < 1) ctas_per_sm = 1;
     if (ctas_per_sm > 8) ctas_per_sm = 8;
@@ -355,7 +337,6 @@ cudaError_t try_launch_cta(const int8_t *logits, void *probs, const RowArgs &a, 
 // Everything the kernel needs besides the caller's tensors lives in this one file-scope device
 // array, which every GPU that loads the library holds until the process exits:
 //   word 0            status word (bounded waits report here)
-//   word 1            row counter of the persistent CTAs
 //   from byte 256 on  the per-head parameter table, kStaticMaxHeads entries
 namespace {
 
@@ -363,6 +344,17 @@ constexpr int kStaticMaxHeads = 256;
 constexpr int kStaticTableOffsetWords = 64;
 constexpr int kStaticWords = kStaticTableOffsetWords + kStaticMaxHeads * (int)(sizeof(hccs::HeadEntry) / 4);
 static __device__ __align__(256) uint32_t g_static_scratch[kStaticWords];
+
+// The table travels to the device as a kernel argument (4 KB by value): no host buffer has to stay alive
+// and nothing is copied from pageable memory, so the call never blocks on earlier work of the stream.
+struct StaticTable {
+    hccs::HeadEntry entry[kStaticMaxHeads];
+};
+__global__ void static_scratch_fill_kernel(uint32_t *scratch, StaticTable table, int num_heads) {
+    if (threadIdx.x == 0) scratch[0] = 0;                         // status word: starts at zero for every call
+    hccs::HeadEntry *dst = reinterpret_cast<hccs::HeadEntry *>(scratch + kStaticTableOffsetWords);
+    for (int h = threadIdx.x; h < num_heads; h += blockDim.x) dst[h] = table.entry[h];
+}
 
 constexpr int kStaticMaxDevices = 64;
 uint32_t *g_static_ptr[kStaticMaxDevices] = {};   // device address of the array, per device
@@ -416,25 +408,24 @@ extern "C" hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *p
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
 
-    // The array keeps whatever the previous call left: rewrite the table, clear the status
-    // word (the launcher clears the row counter).
-    hccs::HeadEntry table[kStaticMaxHeads];
+    // The array keeps whatever the previous call left: a one-CTA kernel on the caller's stream rewrites
+    // the table and clears the status word before the row kernel runs.
+    StaticTable table;
     for (int32_t h = 0; h < num_heads; ++h) {
-        table[h].B = params[h].B;
-        table[h].S = params[h].S;
-        table[h].D = params[h].Dmax;
-        table[h].Drep = (uint32_t)params[h].Dmax * 0x01010101u;
+        table.entry[h].B = params[h].B;
+        table.entry[h].S = params[h].S;
+        table.entry[h].D = params[h].Dmax;
+        table.entry[h].Drep = (uint32_t)params[h].Dmax * 0x01010101u;
     }
     hccs::HeadEntry *d_table = reinterpret_cast<hccs::HeadEntry *>(scratch + kStaticTableOffsetWords);
-    cudaError_t e = cudaMemcpyAsync(d_table, table, sizeof(hccs::HeadEntry) * num_heads,
-                                    cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(scratch, 0, sizeof(uint32_t), stream);
-    if (e != cudaSuccess) { (void)cudaGetLastError(); return HCCS_ERR_CUDA; }
+    static_scratch_fill_kernel<<<1, 256, 0, stream>>>(scratch, table, num_heads);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return HCCS_ERR_CUDA;
 
     hccs::RowArgs a;
     a.table = d_table;
     a.status = scratch;
-    a.row_counter = scratch + 1;
+    a.wait_cycles = hccs::kDefaultWaitCycles;
     a.rows = (int32_t)rows;
     a.H = H;
     a.Lq = Lq;
@@ -465,3 +456,42 @@ extern "C" hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *p
     }
     return HCCS_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Wait-limit probe: the give-up path of the bounded waits, exercised without any copy in flight.
+// ------------------------------------------------------------------------------------------
+namespace hccs {
+
+namespace {
+
+// One CTA of two warps.  Thread 0 initialises an mbarrier that expects one arrival which never comes and
+// waits on it through the helper the production kernels use, with the caller's limit; the wait runs out,
+// the status bit is set and the kernel returns.  In mode 1 a thread of the second warp waits through the
+// abortable helper as well, with a limit sixteen times longer: it leaves because it sees the abort flag.
+__global__ void wait_probe_kernel(uint32_t *status, int mode, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar_word;
+    __shared__ int abort_flag;
+    const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&bar_word);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(1) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    volatile int *abortp = &abort_flag;
+    if (mode == 0) {
+        if (threadIdx.x == 0 && !mbar_wait_bounded(bar, 0, limit_cycles)) atomicOr(status, STATUS_ROW_TMA_TIMEOUT);
+    } else {
+        if (threadIdx.x == 0) (void)mbar_wait_abortable(bar, 0, abortp, status, STATUS_FUSED_TIMEOUT, limit_cycles);
+        if (threadIdx.x == 32) (void)mbar_wait_abortable(bar, 0, abortp, status, STATUS_FUSED_TIMEOUT, limit_cycles * 16);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_wait_probe(uint32_t *status, int mode, long long limit_cycles, cudaStream_t stream) {
+    wait_probe_kernel<<<1, 64, 0, stream>>>(status, mode, limit_cycles);
+    return cudaGetLastError();
+}
+
+}  // namespace hccs

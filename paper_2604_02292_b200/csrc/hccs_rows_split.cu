@@ -12,7 +12,7 @@
 //            r = D - delta = max(x + (D - m), 0)   one viaddmax.s16x2 per split word
 //            so that the score is s = B - S*delta = F + S*r with F = B - S*D (Eq. 2, Eq. 3);
 //            every quantity stays non-negative
-//   stage 4  Z = n_valid*F + S*sum(r)       one three-input add per word (16-bit lane sums)
+//   stage 4  Z = n_valid*F + S*sum(r)       two dot products with ones per word (dp2a, multiply pipe)
 //   stage 5  rho once per row; p = (F*rho' + S*rho'*r) >> 16 with rho' = rho << (1 - OUT_SHIFT)
 // For uint8 output X = s*rho' < 2^24 (s <= Z), and the two elements of a 16-bit pair are normalised by
 // two 32-bit multiply-adds on the pair: the coefficients are split at 8 bits so that every partial
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     // ---- stages 2-4: closeness r = max(x + (D - m), 0) and its row sum
     const int cm = th.D - m;                               // in [-126, 255]
     const uint32_t c2 = prmt((uint32_t)cm, 0, 0x1010u);    // (cm, cm) as 16-bit lanes
-    uint32_t rsum2 = 0;
+    uint32_t racc = 0;
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         if (!chunk_used(v)) continue;
@@ -201,10 +201,10 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         for (int k = CW * v; k < CW * v + CW; ++k) {
             e[k] = __viaddmax_s16x2(e[k], c2, 0u);
             o[k] = __viaddmax_s16x2(o[k], c2, 0u);
-            rsum2 = rsum2 + e[k] + o[k];                   // lane sums stay below 2^16
+            racc = __dp2a_lo(o[k], 0x0101u, __dp2a_lo(e[k], 0x0101u, racc));   // both lanes of both words, on the multiply pipe
         }
     }
-    int rsum = (int)(rsum2 & 0xffffu) + (int)(rsum2 >> 16);
+    int rsum = (int)racc;
 #pragma unroll
     for (int s = G / 2; s; s >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, s);
     // masked keys that were materialised were counted at x = -128
@@ -253,10 +253,12 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
             }
         }
     } else {
-        const int sh = 1 - a.out_shift;                    // 0 or 1 (checked by the launcher)
-        const uint32_t rp = rho << sh;
+        // rho' = rho << (1 - OUT_SHIFT) and p = X >> 16 for the divide; rho' = rho >> OUT_SHIFT (exact: the
+        // leading-bit rho is 255 * 2^(15-k), k <= 14) and p = min(X >> 15, 255) for the leading-bit form, so
+        // that X = s * rho' stays below 2^24 in both (s <= Z < 2^(k+1)); OUT_SHIFT is 0 or 1 (the launcher checks)
+        const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
         const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
-        // Exact divide: X = a1 + b1*r = s*rho' < 2^24 (s <= Z), p = X >> 16.  With a1 = ah*256 + al and
+        // X = a1 + b1*r.  With a1 = ah*256 + al and
         // b1 = bh*256 + bl, X >> 8 = ah + bh*r + ((al + bl*r) >> 8) =: Y < 2^16, and both ah + bh*r and
         // al + bl*r (r <= 127) fit 16 bits: a pair of elements takes two 32-bit multiply-adds on its 16-bit
         // lanes, one byte permute for the carry, one add, and p is the high byte of each lane of Y.
@@ -280,12 +282,11 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                         const uint32_t yo = ro * bh + ah2 + prmt(ro * bl + al2, 0, 0x4341u);
                         out[k] = prmt(ye, yo, 0x7351u);
                     } else {
-                        // the leading-bit reciprocal can overshoot 255: saturate each element
-                        const uint32_t x0 = min(a1 + b1 * (re & 0xffffu), 0x00ffffffu);
-                        const uint32_t x1 = min(a1 + b1 * (ro & 0xffffu), 0x00ffffffu);
-                        const uint32_t x2 = min(a1 + b1 * (re >> 16), 0x00ffffffu);
-                        const uint32_t x3 = min(a1 + b1 * (ro >> 16), 0x00ffffffu);
-                        out[k] = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                        // the leading-bit reciprocal can overshoot: Y saturates at 255*128 + 127 in the add
+                        // itself, and p = Y >> 7 is then bits 7..14 of each lane (bytes 0 and 2 after the shift)
+                        const uint32_t ye = __viaddmin_u16x2(re * bh + ah2, prmt(re * bl + al2, 0, 0x4341u), 0x7fff7fffu);
+                        const uint32_t yo = __viaddmin_u16x2(ro * bh + ah2, prmt(ro * bl + al2, 0, 0x4341u), 0x7fff7fffu);
+                        out[k] = prmt(ye >> 7, yo >> 7, 0x6240u);
                     }
                 }
                 if (!full[v]) {

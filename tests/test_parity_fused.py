@@ -99,19 +99,15 @@ def test_requantisation_corner_cases(hccs, oracle, sh, mults, flags):
     assert_same(got, want, f"fused requant sh={sh} mult={mults} flags={flags}")
 
 
-def test_config5_sampled_heads(hccs, oracle):
-    """The benchmark's fused workload at full size; the oracle recomputes a sample of heads."""
+def test_config5_every_head_slice(hccs, oracle):
+    """The benchmark's fused workload at full size: every one of the 384 (batch, head) slices is
+    recomputed by the oracle (about 40 core-seconds, spread over the host cores)."""
+    import os
     wl = hccs.workloads.make_config(5)
     got = _run(hccs, wl.Q, wl.K, wl.V, wl.theta, wl.requant_mult, wl.requant_shift, wl.n_design)
-    Bt, H, L, d = wl.shape
-    rng = np.random.default_rng(0)
-    heads = sorted(set(int(v) for v in rng.integers(0, Bt * H, size=10)) | {0, Bt * H - 1})
-    g = got.reshape(Bt * H, L, d)
-    for bh in heads:
-        want = oracle.attention(wl.Q, wl.K, wl.V, wl.requant_mult, wl.requant_shift, wl.theta,
-                                bh_range=(bh, bh + 1), threads=1).reshape(Bt * H, L, d)
-        assert_same(g[bh], want[bh], f"config5 head slice {bh}")
-    assert (got != 0x7EADBEEF).all()
+    want = oracle.attention(wl.Q, wl.K, wl.V, wl.requant_mult, wl.requant_shift, wl.theta,
+                            threads=os.cpu_count() or 1)
+    assert_same(got, want, "config5, all head slices")
 
 
 def test_unsupported_shapes_are_refused(hccs):
