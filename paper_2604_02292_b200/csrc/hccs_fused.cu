@@ -62,11 +62,6 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
-__device__ __forceinline__ uint64_t mad_wide_u32(uint32_t a, uint32_t b, uint64_t c) {
-    uint64_t d;
-    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
-    return d;
-}
 __device__ __forceinline__ uint64_t make_u64(uint32_t lo, uint32_t hi) {
     uint64_t d;
     asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
@@ -583,9 +578,16 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const int F = th.B - th.S * th.D;
             const uint32_t Z = (uint32_t)(nv * F + th.S * rs);
             const uint32_t rho = reciprocal<false, CLB>(max(Z, 1u));
-            const uint32_t rp = rho << (1 - a.out_shift);
+            // X = s * rho' = a1 + b1*r < 2^24 with rho' = rho << (1 - OUT_SHIFT) for the divide (p = X >> 16) and
+            // rho' = rho >> OUT_SHIFT for the leading-bit form (p = min(X >> 15, 255); its rho is 255 * 2^(15-k),
+            // k <= 14).  Two keys share a 32-bit multiply-add on 16-bit lanes: with a1 = ah*256 + al and
+            // b1 = b1h*256 + b1l, X >> 8 = ah + b1h*r + ((al + b1l*r) >> 8) < 2^16, and every partial result fits
+            // its lane (r <= 127).  (A 64-bit multiply-add with the keys 24 bits apart needs one multiply per
+            // pair instead of two, but its 64-bit addend costs two more instructions on the integer pipe.)
+            const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
             const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
-            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+            const uint32_t ah2 = (a1 >> 8) * 0x00010001u, al2 = (a1 & 255u) * 0x00010001u;
+            const uint32_t b1h = b1 >> 8, b1l = b1 & 255u;
 
             // ---- phase 3: probabilities from the stored closeness values, in place
             for (int kb = 0; kb < kblocks; ++kb) {
@@ -599,17 +601,17 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     uint32_t o[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
+                        const uint32_t re = prmt(w[k], 0, 0x4240u), ro = prmt(w[k], 0, 0x4341u);   // keys 0, 2 and 1, 3
                         uint32_t q;
                         if (!CLB) {
-                            const uint64_t pe = mad_wide_u32(prmt(w[k], 0, 0x2440u), b1, A);   // keys 0, 2
-                            const uint64_t po = mad_wide_u32(prmt(w[k], 0, 0x3441u), b1, A);   // keys 1, 3
-                            q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                            const uint32_t ye = re * b1h + ah2 + prmt(re * b1l + al2, 0, 0x4341u);
+                            const uint32_t yo = ro * b1h + ah2 + prmt(ro * b1l + al2, 0, 0x4341u);
+                            q = prmt(ye, yo, 0x7351u);
                         } else {
-                            const uint32_t x0 = min(a1 + b1 * (w[k] & 0xffu), 0x00ffffffu);
-                            const uint32_t x1 = min(a1 + b1 * prmt(w[k], 0, 0x4441u), 0x00ffffffu);
-                            const uint32_t x2 = min(a1 + b1 * prmt(w[k], 0, 0x4442u), 0x00ffffffu);
-                            const uint32_t x3 = min(a1 + b1 * (w[k] >> 24), 0x00ffffffu);
-                            q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                            // saturation at 255 folded into the add: Y stops at 255*128 + 127, p = Y >> 7
+                            const uint32_t ye = __viaddmin_u16x2(re * b1h + ah2, prmt(re * b1l + al2, 0, 0x4341u), 0x7fff7fffu);
+                            const uint32_t yo = __viaddmin_u16x2(ro * b1h + ah2, prmt(ro * b1l + al2, 0, 0x4341u), 0x7fff7fffu);
+                            q = prmt(ye >> 7, yo >> 7, 0x6240u);
                         }
                         if (CAUSAL) {
                             const int nb = nv - (kb * kTile + (2 * grp + c) * 16 + 4 * k);
