@@ -203,6 +203,21 @@ int64_t hccs_oracle_requant(int64_t acc, int64_t M, int64_t sh)
 }
 
 /*
+ * int8 output of the fused path: every int32 element of O [B*H, L, d] requantised with its head's
+ * multiplier by the same rounding rule as the logits (hccs_oracle_requant): not in the paper,
+ * which stops at the integer probabilities; the reading is the library's requantisation rule
+ * applied once more.  Mo holds one multiplier per head.
+ */
+void hccs_oracle_requant_output(const int32_t *O, int8_t *out, const int32_t *Mo, int64_t sh,
+                                int64_t BH, int64_t H, int64_t L, int64_t d)
+{
+    int64_t bh, k;
+    for (bh = 0; bh < BH; ++bh)
+        for (k = 0; k < L * d; ++k)
+            out[bh * L * d + k] = (int8_t)hccs_oracle_requant(O[bh * L * d + k], Mo[bh % H], sh);
+}
+
+/*
  * Integer attention for (batch*head) slices [bh_begin, bh_end) and query rows
  * [q_begin, q_end) of each: Q,K,V int8 [Bt,H,L,d]; logits x_ij =
  * requant(sum_d Q[i,d]*K[j,d], M[h], sh); P = HCCS(x_i.) in u8 mode with the

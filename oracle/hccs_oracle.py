@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
             L.hccs_oracle_forward.restype = ctypes.c_int
             L.hccs_oracle_requant.argtypes = [_i64, _i64, _i64]
             L.hccs_oracle_requant.restype = _i64
+            L.hccs_oracle_requant_output.argtypes = [_p, _p, _p, _i64, _i64, _i64, _i64, _i64]
+            L.hccs_oracle_requant_output.restype = None
             L.hccs_oracle_attention.argtypes = [_p, _p, _p, _p, _p, _i64, _p,
                                                 _i64, _i64, _i64, _i64, ctypes.c_int, _i64,
                                                 _i64, _i64, _i64, _i64, _p, _p, _p, _p, _p, _p]
@@ -175,6 +177,17 @@ def attention(Q, K, V, M, sh, params, mode: int = 0, out_shift: int = 0, threads
     if want_intermediates:
         return O, lg, pr
     return O
+
+
+def requant_output(O, Mo, sh: int):
+    """int8 view of an int32 attention output [B,H,L,d]: every element requantised with its head's
+    multiplier Mo[h] and the shift sh by the rule of ``requant``."""
+    O = np.ascontiguousarray(O, dtype=np.int32)
+    Bt, H, Lx, d = O.shape
+    Ma = np.ascontiguousarray(Mo, dtype=np.int32).reshape(H)
+    out = np.zeros(O.shape, dtype=np.int8)
+    lib().hccs_oracle_requant_output(_ptr(O), _ptr(out), _ptr(Ma), int(sh), Bt * H, H, Lx, d)
+    return out
 
 
 def _spread(work, lo, hi, threads):

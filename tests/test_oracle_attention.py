@@ -93,3 +93,29 @@ def test_key_length_mask_equals_attention_over_the_truncated_keys():
                     x = np.array([orc.requant(int(a_), int(M[h]), 12) for a_ in acc], dtype=np.int8)
                     p = orc.forward(x.reshape(1, 1, 1, n), theta[h:h + 1], mode).reshape(n).astype(np.int64)
                     assert np.array_equal(got[b, h, i], (p @ V[b, h, :n].astype(np.int64)).astype(np.int32))
+
+
+def test_output_requantisation_head_index_and_rounding():
+    """int8 output of the fused path: element (b, h, i, c) takes head h's multiplier, and each value is
+    clamp(floor(O*Mo / 2^sh + 1/2), -128, 127), checked with exact fractions on every element of a small
+    tensor that holds the half-way cases, both clamps and all-zero rows."""
+    rng = np.random.default_rng(9)
+    Bt, H, L, d = 2, 3, 5, 4
+    O = rng.integers(-40000, 40001, size=(Bt, H, L, d)).astype(np.int32)
+    sh = 15
+    Mo = np.array([1, 2 ** 14, 173], dtype=np.int32)       # head 1: acc * 2^14 / 2^15 = acc / 2, half-way for odd acc
+    O[0, 1, 0] = (-3, -1, 1, 3)                            # -1.5 -> -1, -0.5 -> 0, 0.5 -> 1, 1.5 -> 2
+    O[1, 2, 1] = (24149, 24150, -24339, -24340)            # last value inside and first beyond each clamp (multiplier 173)
+    O[1, 0, 4] = 0
+    got = orc.requant_output(O, Mo, sh)
+    assert got.dtype == np.int8 and got.shape == O.shape
+    for b in range(Bt):
+        for h in range(H):
+            for i in range(L):
+                for c in range(d):
+                    exact = Fraction(int(O[b, h, i, c]) * int(Mo[h]), 2 ** sh) + Fraction(1, 2)
+                    want = max(-128, min(127, math.floor(exact)))
+                    assert int(got[b, h, i, c]) == want, (b, h, i, c)
+    assert got[0, 1, 0].tolist() == [-1, 0, 1, 2]
+    assert got[1, 2, 1].tolist() == [127, 127, -128, -128]
+    assert (got[1, 0, 4] == 0).all()
