@@ -197,6 +197,21 @@ hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const i
                                        int32_t B, int32_t H, int32_t L, int32_t d,
                                        uint32_t flags, void *cuda_stream);
 
+/*
+ * hccs_attention_fused with an int8 output, for pipelines that stay in int8 after the attention:
+ * O[b,h,i,c] = clamp((acc * out_mult[h] + 2^(out_shift-1)) >> out_shift, -128, 127), acc the int32
+ * accumulator of P.V, i.e. the rounding rule of the logit requantisation applied to the output
+ * (round half up, arithmetic shift, then clamp; exact: computed in 64 bits).
+ *   O          device int8 [B, H, L, d]
+ *   out_mult   HOST int32 [H], each in [0, 2^13);  out_shift in 1..31
+ * Everything else as hccs_attention_fused.  (Not in the paper.)
+ */
+hccs_status_t hccs_attention_fused_i8(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                      const int8_t *V, int8_t *O, const int32_t *out_mult, int32_t out_shift,
+                                      const int32_t *requant_mult, int32_t requant_shift,
+                                      int32_t B, int32_t H, int32_t L, int32_t d,
+                                      uint32_t flags, void *cuda_stream);
+
 /* A bounded grid of candidates for hccs_calibrate: D = D_lo, D_lo + D_step, ... <= D_hi (clipped to
  * 1..127), S likewise (clipped to 0..127), and for each (D, S) the values B = S*D + ceil(256/n),
  * + B_step, ... <= floor(32767/n): every candidate lies in the admissible band (Eq. 11). */

@@ -37,7 +37,7 @@ HCCS_CAUSAL = 4
 
 EXPORTS = ("hccs_create", "hccs_destroy", "hccs_params_check", "hccs_params_upload", "hccs_forward",
            "hccs_forward_keylen", "hccs_forward_host",
-           "hccs_attention_fused", "hccs_attention_fused_keylen", "hccs_attention_fused_f32", "hccs_device_status", "hccs_last_cuda_error", "hccs_status_string",
+           "hccs_attention_fused", "hccs_attention_fused_keylen", "hccs_attention_fused_f32", "hccs_attention_fused_i8", "hccs_device_status", "hccs_last_cuda_error", "hccs_status_string",
            "hccs_launch_count", "hccs_forward_static_scratch", "hccs_calibrate", "hccs_debug_wait_timeout")
 
 _vp, _i32, _u32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32
@@ -65,6 +65,9 @@ _lib.hccs_attention_fused_keylen.restype = ctypes.c_int
 _lib.hccs_attention_fused_f32.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
                                           _u32, _vp]
 _lib.hccs_attention_fused_f32.restype = ctypes.c_int
+_lib.hccs_attention_fused_i8.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i32, _i32, _i32, _i32, _i32,
+                                         _u32, _vp]
+_lib.hccs_attention_fused_i8.restype = ctypes.c_int
 _lib.hccs_device_status.argtypes = [_vp, ctypes.POINTER(_u32), _vp]
 _lib.hccs_device_status.restype = ctypes.c_int
 _lib.hccs_last_cuda_error.argtypes = [_vp]
@@ -251,6 +254,23 @@ class Context:
                                            int(requant_shift), B, H, L, d, int(flags), _stream_ptr(stream))
         if st != HCCS_OK:
             raise HccsError(st, "hccs_attention_fused_f32")
+
+    # -- hccs_attention_fused_i8
+    def hccs_attention_fused_i8(self, Q, K, V, O, out_mult, out_shift: int, requant_mult, requant_shift: int,
+                                flags: int = 0, stream=None) -> None:
+        B, H, L, d = Q.shape
+        for name, t in (("Q", Q), ("K", K), ("V", V)):
+            _check_tensor(t, name, 1, Q.shape)
+        _check_tensor(O, "O", 1, Q.shape)
+        mult = np.ascontiguousarray(requant_mult, dtype=np.int32).reshape(-1)
+        omult = np.ascontiguousarray(out_mult, dtype=np.int32).reshape(-1)
+        if mult.size != H or omult.size != H:
+            raise ValueError("requant_mult and out_mult must have H entries")
+        st = _lib.hccs_attention_fused_i8(self._h, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), omult.ctypes.data_as(_vp),
+                                          int(out_shift), mult.ctypes.data_as(_vp), int(requant_shift), B, H, L, d,
+                                          int(flags), _stream_ptr(stream))
+        if st != HCCS_OK:
+            raise HccsError(st, "hccs_attention_fused_i8")
 
     # -- hccs_device_status / hccs_last_cuda_error / hccs_launch_count
     def hccs_device_status(self, stream=None) -> int:

@@ -342,9 +342,11 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
     return HCCS_OK;
 }
 
-// Shared by the int32 and the fp32 entry points: out_scale == NULL means int32 output.
+// Shared by the int32, fp32 and int8 entry points: out_scale != NULL means fp32 output, out_mult != NULL
+// int8 output, neither int32 output.
 static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K, const int8_t *V, void *O,
-                                  const float *out_scale, const int32_t *key_len, const int32_t *requant_mult,
+                                  const float *out_scale, const int32_t *out_mult, int32_t out_shift,
+                                  const int32_t *key_len, const int32_t *requant_mult,
                                   int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
                                   uint32_t flags, void *cuda_stream) {
     if (!ctx || B < 0 || H < 0 || L < 0 || d < 0) return HCCS_ERR_INVALID_ARG;
@@ -355,6 +357,11 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     if (requant_shift < 1 || requant_shift > 31) return HCCS_ERR_INVALID_ARG;
     for (int32_t h = 0; h < H; ++h)
         if (requant_mult[h] < 0 || requant_mult[h] >= (1 << 13)) return HCCS_ERR_INVALID_ARG;
+    if (out_mult) {
+        if (out_shift < 1 || out_shift > 31) return HCCS_ERR_INVALID_ARG;
+        for (int32_t h = 0; h < H; ++h)
+            if (out_mult[h] < 0 || out_mult[h] >= (1 << 13)) return HCCS_ERR_INVALID_ARG;
+    }
     // the kernel requantises with the multiplier pre-shifted by 32 - requant_shift bits
     for (int32_t h = 0; h < H; ++h)
         if ((int64_t)requant_mult[h] << (32 - requant_shift) >= (1ll << 31)) return HCCS_ERR_UNSUPPORTED;
@@ -369,7 +376,7 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     // Per head: {multiplier, and for shifts up to 24 the constants of the single-multiply
     // requantisation: multiplier << k, offset, -lo, hi - lo} (see hccs_fused.cu, phase 1), then the
-    // fp32 output scale, a spare word and 1 / multiplier as a double; eight 32-bit words per head.
+    // fp32 output scale, the int8 output multiplier and 1 / multiplier as a double; eight 32-bit words per head.
     // The words are built on the stack and go up only when they differ from what the device table
     // already holds (the usual case is the same multipliers call after call): then nothing is copied
     // and the host never waits for an earlier call's copy.
@@ -381,7 +388,8 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
         const int64_t M = requant_mult[h];
         int32_t *e = words + 8 * h;
         e[0] = (int32_t)M;
-        e[1] = e[2] = e[3] = e[5] = e[6] = e[7] = 0;
+        e[1] = e[2] = e[3] = e[6] = e[7] = 0;
+        e[5] = out_mult ? out_mult[h] : 0;
         const float scale = out_scale ? out_scale[h] : 1.0f;
         memcpy(&e[4], &scale, sizeof(float));
         const double inv_m = M > 0 ? 1.0 / (double)M : 0.0;      // words 6 and 7
@@ -430,7 +438,8 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     a.requant_mult = ctx->d_mult;
     a.status = ctx->d_status;
     a.wait_cycles = hccs::kDefaultWaitCycles;
-    a.out_f32 = out_scale ? 1 : 0;
+    a.out_mode = out_scale ? 1 : (out_mult ? 2 : 0);
+    a.out_requant_shift = out_mult ? out_shift : 1;
     a.key_len = key_len;
     a.requant_shift = requant_shift;
     a.B = B; a.H = H; a.L = L; a.d = d;
@@ -444,7 +453,7 @@ hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_
                                    const int8_t *V, int32_t *O, const int32_t *requant_mult,
                                    int32_t requant_shift, int32_t B, int32_t H, int32_t L, int32_t d,
                                    uint32_t flags, void *cuda_stream) {
-    return fused_common(ctx, Q, K, V, O, nullptr, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+    return fused_common(ctx, Q, K, V, O, nullptr, nullptr, 0, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
 }
 
 hccs_status_t hccs_attention_fused_keylen(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
@@ -453,7 +462,7 @@ hccs_status_t hccs_attention_fused_keylen(hccs_ctx_t *ctx, const int8_t *Q, cons
                                           int32_t B, int32_t H, int32_t L, int32_t d,
                                           uint32_t flags, void *cuda_stream) {
     if (!key_len && (int64_t)B * H * L * d != 0) return HCCS_ERR_INVALID_ARG;
-    return fused_common(ctx, Q, K, V, O, nullptr, key_len, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+    return fused_common(ctx, Q, K, V, O, nullptr, nullptr, 0, key_len, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
 }
 
 hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
@@ -462,7 +471,16 @@ hccs_status_t hccs_attention_fused_f32(hccs_ctx_t *ctx, const int8_t *Q, const i
                                        int32_t B, int32_t H, int32_t L, int32_t d,
                                        uint32_t flags, void *cuda_stream) {
     if (!out_scale) return HCCS_ERR_INVALID_ARG;
-    return fused_common(ctx, Q, K, V, O, out_scale, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+    return fused_common(ctx, Q, K, V, O, out_scale, nullptr, 0, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
+}
+
+hccs_status_t hccs_attention_fused_i8(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
+                                      const int8_t *V, int8_t *O, const int32_t *out_mult, int32_t out_shift,
+                                      const int32_t *requant_mult, int32_t requant_shift,
+                                      int32_t B, int32_t H, int32_t L, int32_t d,
+                                      uint32_t flags, void *cuda_stream) {
+    if (!out_mult) return HCCS_ERR_INVALID_ARG;
+    return fused_common(ctx, Q, K, V, O, nullptr, out_mult, out_shift, nullptr, requant_mult, requant_shift, B, H, L, d, flags, cuda_stream);
 }
 
 hccs_status_t hccs_device_status(hccs_ctx_t *ctx, uint32_t *word, void *cuda_stream) {

@@ -652,25 +652,53 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 uint32_t acc[kCols];
                 if constexpr (kCols == 16) tmem_ld16(tmem + lane_addr + kTmemO + grp * kCols, acc);
                 else tmem_ld32(tmem + lane_addr + kTmemO + grp * kCols, acc);
-                if (a.out_f32) {                                  // optional dequantised view of O
+                if (a.out_mode == 1) {                            // optional dequantised view of O
 #pragma unroll
                     for (int g = 0; g < kCols; ++g) acc[g] = __float_as_uint(__int2float_rn((int)acc[g]) * out_scale);
                 }
-                // column c of the tile sits in box c / 32, 16-byte chunk (c % 32) / 4 of its row
                 const int c0 = grp * kCols;
-                uint8_t *o_stage = panel + (c0 >> 5) * kOBoxBytes + t * 128;
+                if (a.out_mode == 2) {
+                    // int8 output: every accumulator requantised with the head's output multiplier by the rule
+                    // of the logits, clamp((acc*Mo + 2^(sh-1)) >> sh, -128, 127), in 64 bits (a handful of
+                    // values per thread and tile); the tile is staged as plain rows of D bytes
+                    const int32_t out_mult = a.requant_mult[8 * head + 5];
+                    const int64_t round = (int64_t)1 << (a.out_requant_shift - 1);
+                    uint32_t packed[kCols / 4];
 #pragma unroll
-                for (int g = 0; g < kCols / 4; ++g)
-                    *reinterpret_cast<uint4 *>(o_stage + (((((c0 & 31) >> 2) + g) ^ swz) << 4)) =
-                        make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
+                    for (int g = 0; g < kCols / 4; ++g) {
+                        int32_t x[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int64_t v = mad_wide_s32((int32_t)acc[4 * g + e], out_mult, round) >> a.out_requant_shift;
+                            x[e] = (int32_t)min(max(v, (int64_t)-128), (int64_t)127);
+                        }
+                        packed[g] = cvt_pack_s8(x[1], x[0], cvt_pack_s8(x[3], x[2], 0u));
+                    }
+                    uint8_t *o_stage = panel + t * D + c0;
+#pragma unroll
+                    for (int g = 0; g < kCols / 16; ++g)
+                        *reinterpret_cast<uint4 *>(o_stage + 16 * g) =
+                            make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
+                } else {
+                    // column c of the tile sits in box c / 32, 16-byte chunk (c % 32) / 4 of its row
+                    uint8_t *o_stage = panel + (c0 >> 5) * kOBoxBytes + t * 128;
+#pragma unroll
+                    for (int g = 0; g < kCols / 4; ++g)
+                        *reinterpret_cast<uint4 *>(o_stage + (((((c0 & 31) >> 2) + g) ^ swz) << 4)) =
+                            make_uint4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
+                }
                 tcgen05_fence_before();
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             if (tid == 0) leave_flag = *abortp;                   // one reader, so that all row threads agree
             asm volatile("bar.sync 1, 512;" ::: "memory");
             if (tid == 0 && !*(volatile int *)&leave_flag) {
+                if (a.out_mode == 2) {
+                    tma_store_3d(&map_o, 0, q0, bh, s_p);          // one box of 128 rows x D bytes
+                } else {
 #pragma unroll
-                for (int b = 0; b < D / 32; ++b) tma_store_3d(&map_o, 32 * b, q0, bh, s_p + b * kOBoxBytes);
+                    for (int b = 0; b < D / 32; ++b) tma_store_3d(&map_o, 32 * b, q0, bh, s_p + b * kOBoxBytes);
+                }
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
             // leave the loop together (the flag was sampled once, before the barrier above)
@@ -735,6 +763,19 @@ bool make_output_map(CUtensorMap *map, const void *ptr, uint64_t heads, uint64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// O as [B*H][L][d] bytes (int8 output), one box of 128 rows x d bytes, no swizzle.
+bool make_output_map_i8(CUtensorMap *map, const void *ptr, uint64_t heads, uint64_t L, uint32_t d) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)L, (cuuint64_t)heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)d, (cuuint64_t)d * L};
+    const cuuint32_t box[3] = {(cuuint32_t)d, (cuuint32_t)kTile, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, bool CLB, bool CAUSAL>
 cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mo,
                            const FusedArgs &a, cudaStream_t st) {
@@ -766,8 +807,10 @@ cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *laun
     CUtensorMap mq, mk, mv, mo;
     const uint64_t rows = (uint64_t)a.B * a.H * a.L;
     if (!fused_shape_supported(a.L, a.d)) return cudaErrorInvalidValue;
-    if (!make_tile_map(&mq, a.Q, rows, a.d) || !make_tile_map(&mk, a.K, rows, a.d) || !make_tile_map(&mv, a.V, rows, a.d) ||
-        !make_output_map(&mo, a.O, (uint64_t)a.B * a.H, (uint64_t)a.L, a.d))
+    if (!make_tile_map(&mq, a.Q, rows, a.d) || !make_tile_map(&mk, a.K, rows, a.d) || !make_tile_map(&mv, a.V, rows, a.d))
+        return cudaErrorInvalidValue;
+    if (!(a.out_mode == 2 ? make_output_map_i8(&mo, a.O, (uint64_t)a.B * a.H, (uint64_t)a.L, a.d)
+                          : make_output_map(&mo, a.O, (uint64_t)a.B * a.H, (uint64_t)a.L, a.d)))
         return cudaErrorInvalidValue;
     cudaError_t e;
     // the masked instantiation also serves L that is no multiple of 128 (padding keys in the last block)

@@ -46,10 +46,11 @@ enum : uint32_t {
 
 struct FusedArgs {
     const int8_t *Q, *K, *V;
-    void *O;                       // int32 [B,H,L,d], or float when out_f32
+    void *O;                       // int32 [B,H,L,d]; float when out_mode == 1; int8 when out_mode == 2
     const HeadEntry *table;
     const int32_t *requant_mult;   // device, 8 words per head: see fused_common in hccs_api.cu
-    int32_t out_f32;               // 1: O = float(acc) * scale_h
+    int32_t out_mode;              // 0: int32 accumulators; 1: float(acc) * scale_h; 2: acc requantised to int8
+    int32_t out_requant_shift;     // out_mode 2: shift of the output requantisation (multipliers: word 5 of the table)
     const int32_t *key_len;        // device, one entry per batch entry, or NULL: keys beyond key_len[b] are padding
     uint32_t *status;
     long long wait_cycles;         // limit of every device-side wait, in SM clock cycles

@@ -176,3 +176,39 @@ def test_key_length_mask(hccs, oracle, d, L, flags, sh):
     want = oracle.attention(Q, K, V, mult, sh, theta, oracle_mode(oracle, flags), threads=16, key_len=key_len)
     assert_same(O.cpu().numpy(), want, f"fused key_len d={d} L={L} flags={flags} sh={sh}")
     ctx.close()
+
+
+@pytest.mark.parametrize("shape,flags", [((2, 3, 333, 64), 0), ((2, 3, 333, 64), 4), ((1, 2, 1024, 64), 2),
+                                         ((1, 2, 200, 128), 0), ((2, 2, 512, 128), 6)])
+def test_int8_output(hccs, oracle, shape, flags):
+    """hccs_attention_fused_i8: the int32 result requantised per head, bit for bit against the oracle's
+    output requantisation of the oracle's attention; multipliers chosen so that both clamps are hit."""
+    import torch
+    rng = np.random.default_rng(5000 + shape[2] + flags)
+    Bt, H, L, d = shape
+    Q, K, V = _rand_qkv(rng, shape, -128, 128)
+    n_design = max(L, 512)
+    theta = hccs.workloads.sample_theta(rng, H, n_design)
+    mult = (rng.integers(768, 3841, size=H) * 64 // d).astype(np.int32)
+    out_mult = rng.integers(100, 8192, size=H).astype(np.int32)
+    out_mult[0] = 8191
+    acc = oracle.attention(Q, K, V, mult, 20, theta, oracle_mode(oracle, flags), threads=8)
+    # a shift that puts the largest accumulator of head 0 near 300: both clamps and the middle are reached
+    out_sh = int(min(31, max(1, np.floor(np.log2(max(int(np.abs(acc[:, 0]).max()), 1) * 8191 / 300.0)))))
+    ctx = hccs.Context(0)
+    ctx.hccs_params_upload(theta, n_design)
+    dQ, dK, dV = (torch.from_numpy(a).cuda() for a in (Q, K, V))
+    O = torch.full(shape, 0x5A, dtype=torch.int8, device="cuda")
+    ctx.hccs_attention_fused_i8(dQ, dK, dV, O, out_mult, out_sh, mult, 20, flags)
+    torch.cuda.synchronize()
+    assert ctx.hccs_device_status() == 0
+    want = oracle.requant_output(acc, out_mult, out_sh)
+    if np.abs(acc[:, 0]).max() > 300:       # (1024 keys of full-range logits give all-zero uint8 probabilities)
+        assert (want == 127).any() and (want == -128).any() and (np.abs(want.astype(np.int32)) < 100).any()
+    assert_same(O.cpu().numpy(), want, f"fused int8 output {shape} flags={flags}")
+    # bad arguments are refused before anything is launched
+    for om, osh in ((out_mult, 0), (out_mult, 32), (np.full(H, 8192, np.int32), 10), (np.full(H, -1, np.int32), 10)):
+        with pytest.raises(hccs.HccsError) as ei:
+            ctx.hccs_attention_fused_i8(dQ, dK, dV, O, om, osh, mult, 20, flags)
+        assert ei.value.status == hccs.HCCS_ERR_INVALID_ARG
+    ctx.close()
