@@ -161,10 +161,10 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
  *   O             device int32 [B, H, L, d]
  *   requant_mult  HOST int32 [H], each in [0, 2^13) and below 2^(requant_shift-1); requant_shift in 1..31
  *   flags         HCCS_RECIP_CLB and HCCS_CAUSAL are honoured; HCCS_OUT_U16 is HCCS_ERR_UNSUPPORTED
- * Supported shapes: d == 64 with 1 <= L <= 1024, or d == 128 with 1 <= L <= 512 (K, V and the
- * 128 x L probability panel share one SM's shared memory); L <= n_design, pointers 16-byte
- * aligned; anything else returns HCCS_ERR_UNSUPPORTED.  The logits and probabilities
- * never leave the chip.
+ * Supported shapes: d == 64 or d == 128 with 1 <= L <= 1024 (the 128 x L probability panel stays in
+ * one SM's shared memory; for d == 128 beyond 512 keys K and V stream through a ring of buffers
+ * beside it); L <= n_design, pointers 16-byte aligned; anything else returns HCCS_ERR_UNSUPPORTED.
+ * The logits and probabilities never leave the chip.
  */
 hccs_status_t hccs_attention_fused(hccs_ctx_t *ctx, const int8_t *Q, const int8_t *K,
                                    const int8_t *V, int32_t *O, const int32_t *requant_mult,

@@ -168,9 +168,18 @@ struct FusedSmemBarriers {
     uint64_t s_free[kSBufs];
     uint64_t p_ready[kMaxBlocks];   // block kb of the probability panel is complete
     uint64_t o_full;
+    uint64_t ring_full[4];          // ring mode: the copy into slot s has landed
+    uint64_t ring_free[4];          // ring mode: every MMA that reads slot s has completed
 };
 
-template <int D, bool CLB, bool CAUSAL>
+// RING (d = 128 with more than 512 keys): K, V and the panel no longer fit the SM together, so the K blocks of
+// the first round, the K blocks of the second round and the V blocks of a tile stream, in that order, through
+// a ring of four 16 KB slots.  Load number j (counted over all tiles of the CTA) uses slot j % 4 for the
+// (j / 4)-th time; every role derives slot and phase parities from j alone.  A slot is handed back by a
+// tcgen05.commit behind the MMAs that read it.
+constexpr int kRingSlots = 4;
+
+template <int D, bool CLB, bool CAUSAL, bool RING = false>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
@@ -195,8 +204,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     const uint32_t s_q = base;                                            // Q tile
     const uint32_t s_kpre = s_q + kTileBytes;                             // K blocks 0 and 1 (prefetched)
     const uint32_t s_kv = s_kpre + 2 * kTileBytes;                        // K blocks 2.., later all V blocks
-    const uint32_t s_p = s_kv + (uint32_t)nblk * kTileBytes;              // logit / probability panel
-    uint8_t *panel = gen_base + 3 * kTileBytes + (size_t)nblk * kTileBytes;
+    const uint32_t s_ring = s_q + kTileBytes;                             // ring mode: the four K / V slots
+    const uint32_t s_p = RING ? s_ring + kRingSlots * kTileBytes : s_kv + (uint32_t)nblk * kTileBytes;   // logit / probability panel
+    uint8_t *panel = gen_base + (RING ? (1 + kRingSlots) * kTileBytes : 3 * kTileBytes + (size_t)nblk * kTileBytes);
+    const int ring_stages = (two_rounds ? 2 : 1) + 1;    // K once per round of the first contraction, then V
     auto k_slot = [&](int kb) { return kb < 2 ? s_kpre + kb * kTileBytes : s_kv + kb * kTileBytes; };
 
     if (tid == 0) {
@@ -211,6 +222,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         }
         for (int i = 0; i < kMaxBlocks; ++i) mbar_init(smem_u32(&bars.p_ready[i]), kRowThreads);
         mbar_init(smem_u32(&bars.o_full), 1);
+        for (int i = 0; i < kRingSlots; ++i) {
+            mbar_init(smem_u32(&bars.ring_full[i]), 1);
+            mbar_init(smem_u32(&bars.ring_free[i]), 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -264,6 +279,32 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     load_tile(k_slot(kb), &map_k, bh * a.L + kb * kTile, smem_u32(&bars.k_full[kb]));
                 }
             };
+            if constexpr (RING) {
+                // loads in ring order; this thread takes the even or the odd ones (slots 0, 2 or 1, 3)
+                uint32_t base_j = 0;
+                for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                    const int bh = tile / nblk, qt = tile % nblk;
+                    const int kblocks = blocks_of(tile);
+                    if (me == 0) {
+                        // Q is read by both rounds of the first contraction: the previous tile's must be complete
+                        if (it > 0) ok = mbar_wait(smem_u32(&bars.k_done), (it - 1) & 1, abortp, a.status, a.wait_cycles);
+                        if (!ok) break;
+                        load_tile(s_q, &map_q, bh * a.L + qt * kTile, smem_u32(&bars.q_full));
+                    }
+                    for (int st = 0; ok && st < ring_stages; ++st) {
+                        for (int kb = 0; kb < kblocks; ++kb) {
+                            const uint32_t j = base_j + (uint32_t)(st * kblocks + kb);
+                            if ((int)(j & 1u) != me) continue;
+                            const uint32_t slot = j % kRingSlots, use = j / kRingSlots;
+                            if (use > 0) ok = mbar_wait(smem_u32(&bars.ring_free[slot]), (use - 1) & 1, abortp, a.status, a.wait_cycles);
+                            if (!ok) break;
+                            load_tile(s_ring + slot * kTileBytes, st + 1 < ring_stages ? &map_k : &map_v, bh * a.L + kb * kTile,
+                                      smem_u32(&bars.ring_full[slot]));
+                        }
+                    }
+                    base_j += (uint32_t)(ring_stages * kblocks);
+                }
+            } else {
             if (me == 0 && (int)blockIdx.x < num_tiles) prefetch(blockIdx.x);
             for (int tile = blockIdx.x, it = 0; ok && tile < num_tiles; tile += gridDim.x, ++it) {
                 const int bh = tile / nblk;
@@ -285,6 +326,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     if (kb == 0 && tile + (int)gridDim.x < num_tiles) prefetch(tile + gridDim.x);
                 }
             }
+            }   // resident K and V
         }
     } else if (warp == kQkWarp || warp == kQk2Warp) {
         // ===================================================== first contraction: S = Q . K^T, block by block.
@@ -296,6 +338,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             uint32_t k_par = 0;                          // bit kb = parity of this tile's phase of k_full[kb]
             uint32_t g = 0;                              // blocks issued so far by both issuers
             uint32_t s_buf = 0, s_cyc = 0;               // = g % kSBufs, g / kSBufs: S buffer of block g and its use
+            uint32_t ring_base = 0;                      // ring mode: load number of this tile's first block
             // descriptors differ only in the start address field (address >> 4): low word + offset
             const uint64_t dq = smem_desc(s_q, 16, 512, kSwizzle64);
             const uint64_t dk = smem_desc(s_kpre, 16, 512, kSwizzle64);
@@ -318,12 +361,21 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         if (cyc > 0) ok = mbar_wait(smem_u32(&bars.s_free[sb]), (cyc - 1) & 1, abortp, a.status, a.wait_cycles);
                         // the K block's copy must have landed: in the second round too, where the
                         // block may fall to the issuer that did not wait for it in the first
-                        if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status, a.wait_cycles);
+                        uint32_t koff;                        // the K block's distance from s_kpre, in 16-byte units
+                        uint32_t ring_slot = 0;
+                        if constexpr (RING) {
+                            const uint32_t j = ring_base + (uint32_t)(round * kblocks + kb);
+                            ring_slot = j % kRingSlots;
+                            if (ok) ok = mbar_wait(smem_u32(&bars.ring_full[ring_slot]), (j / kRingSlots) & 1, abortp, a.status, a.wait_cycles);
+                            koff = (ring_slot * kTileBytes) >> 4;          // s_ring is where s_kpre is
+                        } else {
+                            if (ok) ok = mbar_wait(smem_u32(&bars.k_full[kb]), (k_par >> kb) & 1, abortp, a.status, a.wait_cycles);
+                            // K block kb sits (kb < 2 ? kb : kb + 2) tiles above the first prefetch slot
+                            koff = (uint32_t)((kb < 2 ? kb : kb + 2) * kTileBytes) >> 4;
+                        }
                         if (!ok) break;
                         tcgen05_fence_after();
-                        // K block kb sits (kb < 2 ? kb : kb + 2) tiles above the first prefetch slot;
                         // two k-steps of 32 per 64-byte half of d
-                        const uint32_t koff = (uint32_t)((kb < 2 ? kb : kb + 2) * kTileBytes) >> 4;
 #pragma unroll
                         for (int h = 0; h < kHalves; ++h)
 #pragma unroll
@@ -333,10 +385,12 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                                                kIdescQK, (h | ks) != 0);
                             }
                         tcgen05_commit(smem_u32(&bars.s_full[sb]));
+                        if constexpr (RING) tcgen05_commit(smem_u32(&bars.ring_free[ring_slot]));   // the slot goes back
                     }
                 }
                 if (!ok) break;
                 k_par ^= (1u << kblocks) - 1u;               // every k_full[kb < kblocks] completed one phase
+                ring_base += (uint32_t)(ring_stages * kblocks);
                 tcgen05_commit(smem_u32(&bars.k_done));      // both issuers: the barrier counts two
             }
         }
@@ -346,8 +400,9 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         if (lane == 0) {
             bool ok = true;
             uint32_t p_par = 0;                          // bit kb = parity of the next use of p_ready[kb] and v_full[kb]
+            uint32_t ring_base = 0;                      // ring mode: load number of this tile's first block
             const uint64_t dp = smem_desc(s_p, 16, 1024, kSwizzle128);
-            const uint64_t dv = smem_desc(s_kv, 512, 512, kSwizzle64);
+            const uint64_t dv = smem_desc(RING ? s_ring : s_kv, 512, 512, kSwizzle64);
             const uint32_t dp_lo = (uint32_t)dp, dp_hi = (uint32_t)(dp >> 32);
             const uint32_t dv_lo = (uint32_t)dv, dv_hi = (uint32_t)(dv >> 32);
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
@@ -355,7 +410,16 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                 for (int kb = 0; kb < kMaxBlocks; ++kb) {
                     if (kb >= kblocks) break;
-                    ok = mbar_wait(smem_u32(&bars.v_full[kb]), (p_par >> kb) & 1, abortp, a.status, a.wait_cycles);
+                    uint32_t vbase = (uint32_t)(kb * kTileBytes) >> 4;     // the V block's distance from the descriptor's base, in 16-byte units
+                    uint32_t ring_slot = 0;
+                    if constexpr (RING) {
+                        const uint32_t j = ring_base + (uint32_t)((ring_stages - 1) * kblocks + kb);
+                        ring_slot = j % kRingSlots;
+                        ok = mbar_wait(smem_u32(&bars.ring_full[ring_slot]), (j / kRingSlots) & 1, abortp, a.status, a.wait_cycles);
+                        vbase = (ring_slot * kTileBytes) >> 4;
+                    } else {
+                        ok = mbar_wait(smem_u32(&bars.v_full[kb]), (p_par >> kb) & 1, abortp, a.status, a.wait_cycles);
+                    }
                     if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[kb]), (p_par >> kb) & 1, abortp, a.status, a.wait_cycles);
                     if (!ok) break;
                     p_par ^= 1u << kb;
@@ -365,13 +429,15 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         const uint32_t poff = (uint32_t)(kb * kPanelBlockBytes + ks * 32) >> 4;
 #pragma unroll
                         for (int h = 0; h < kHalves; ++h) {      // 64 output columns per half tile of V
-                            const uint32_t voff = (uint32_t)(kb * kTileBytes + h * kHalfBytes + ks * 32 * kHalf) >> 4;
+                            const uint32_t voff = vbase + ((uint32_t)(h * kHalfBytes + ks * 32 * kHalf) >> 4);
                             tcgen05_mma_i8(tmem + kTmemO + h * kHalf, make_u64(dp_lo + poff, dp_hi), make_u64(dv_lo + voff, dv_hi),
                                            kIdescPV, (kb | ks) != 0);
                         }
                     }
+                    if constexpr (RING) tcgen05_commit(smem_u32(&bars.ring_free[ring_slot]));   // the slot goes back
                 }
                 if (!ok) break;
+                ring_base += (uint32_t)(ring_stages * kblocks);
                 tcgen05_commit(smem_u32(&bars.o_full));
             }
         }
@@ -776,15 +842,16 @@ bool make_output_map_i8(CUtensorMap *map, const void *ptr, uint64_t heads, uint6
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool CLB, bool CAUSAL>
+template <int D, bool CLB, bool CAUSAL, bool RING = false>
 cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mo,
                            const FusedArgs &a, cudaStream_t st) {
     const int nblk = (a.L + kTile - 1) / kTile;
     constexpr size_t kTileBytes = (size_t)kTile * D;
     size_t panel = (size_t)kTile * nblk * kTile;
     if (panel < (D / 32) * (size_t)kOBoxBytes) panel = (D / 32) * (size_t)kOBoxBytes;   // the staged O boxes reuse the panel
-    const size_t smem = 1024 + 3 * kTileBytes + (size_t)nblk * kTileBytes + panel;
-    auto kernel = fused_attention_kernel<D, CLB, CAUSAL>;
+    // resident: Q, two prefetch slots, a slot per K / V block, the panel; ring: Q, four slots, the panel
+    const size_t smem = 1024 + (RING ? (1 + kRingSlots) * kTileBytes : 3 * kTileBytes + (size_t)nblk * kTileBytes) + panel;
+    auto kernel = fused_attention_kernel<D, CLB, CAUSAL, RING>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t tiles = (int64_t)a.B * a.H * nblk;
@@ -798,9 +865,10 @@ cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const C
 
 }  // namespace
 
-// d = 64 with up to 1024 keys, d = 128 with up to 512 (K, V and the panel share the SM's shared memory).
+// d = 64 or 128 with up to 1024 keys (d = 128 beyond 512 keys streams K and V through a ring: K, V and the
+// panel no longer fit the SM's shared memory together).
 bool fused_shape_supported(int32_t L, int32_t d) {
-    return L >= 1 && ((d == 64 && L <= kTile * kMaxBlocks) || (d == 128 && L <= kTile * kMaxBlocks / 2));
+    return L >= 1 && L <= kTile * kMaxBlocks && (d == 64 || d == 128);
 }
 
 cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *launches) {
@@ -822,11 +890,16 @@ cudaError_t launch_fused(const FusedArgs &a, cudaStream_t stream, uint64_t *laun
         else if (clb && !causal) e = launch_variant<64, true, false>(mq, mk, mv, mo, a, stream);
         else if (!clb && causal) e = launch_variant<64, false, true>(mq, mk, mv, mo, a, stream);
         else e = launch_variant<64, true, true>(mq, mk, mv, mo, a, stream);
-    } else {
+    } else if (a.L <= kTile * kMaxBlocks / 2) {
         if (!clb && !causal) e = launch_variant<128, false, false>(mq, mk, mv, mo, a, stream);
         else if (clb && !causal) e = launch_variant<128, true, false>(mq, mk, mv, mo, a, stream);
         else if (!clb && causal) e = launch_variant<128, false, true>(mq, mk, mv, mo, a, stream);
         else e = launch_variant<128, true, true>(mq, mk, mv, mo, a, stream);
+    } else {
+        if (!clb && !causal) e = launch_variant<128, false, false, true>(mq, mk, mv, mo, a, stream);
+        else if (clb && !causal) e = launch_variant<128, true, false, true>(mq, mk, mv, mo, a, stream);
+        else if (!clb && causal) e = launch_variant<128, false, true, true>(mq, mk, mv, mo, a, stream);
+        else e = launch_variant<128, true, true, true>(mq, mk, mv, mo, a, stream);
     }
     if (e == cudaSuccess && launches) ++*launches;
     return e;

@@ -54,6 +54,51 @@ def test_head_dimension_128(hccs, oracle, L, flags):
     assert_same(got, want, f"fused d=128 L={L} flags={flags}")
 
 
+@pytest.mark.parametrize("L", [513, 640, 1000, 1024])
+@pytest.mark.parametrize("flags", [0, 4, 6])
+def test_head_dimension_128_beyond_512_keys(hccs, oracle, L, flags):
+    """d = 128 with more than 512 keys: K and V stream through a ring of four slots (K twice, for the two
+    rounds of the first contraction, then V).  More tiles than SMs, so that the ring runs across tiles."""
+    rng = np.random.default_rng(4200 + L + flags)
+    Bt, H, d = 7, 3, 128
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d), -128, 128)
+    theta = hccs.workloads.sample_theta(rng, H, 1024)
+    mult = rng.integers(150, 700, size=H).astype(np.int32)
+    got = _run(hccs, Q, K, V, theta, mult, 20, 1024, flags)
+    want = oracle.attention(Q, K, V, mult, 20, theta, oracle_mode(oracle, flags), threads=8)
+    assert_same(got, want, f"fused d=128 L={L} flags={flags}")
+
+
+def test_head_dimension_128_ring_key_lengths_and_wide_shift(hccs, oracle):
+    """The ring with per-batch key lengths (tiles use different numbers of key blocks, also zero keys) and
+    with the single-round requantisation flow of shifts above 24."""
+    import torch
+    rng = np.random.default_rng(4300)
+    Bt, H, L, d = 6, 2, 900, 128
+    Q, K, V = _rand_qkv(rng, (Bt, H, L, d))
+    theta = hccs.workloads.sample_theta(rng, H, 1024)
+    mult = rng.integers(300, 900, size=H).astype(np.int32)
+    key_len = np.array([900, 0, 1, 513, 129, 640], dtype=np.int32)
+    ctx = hccs.Context(0)
+    ctx.hccs_params_upload(theta, 1024)
+    dQ, dK, dV = (torch.from_numpy(a).cuda() for a in (Q, K, V))
+    for flags in (0, 4):
+        O = torch.full(Q.shape, 0x7EADBEEF, dtype=torch.int32, device="cuda")
+        ctx.hccs_attention_fused_keylen(dQ, dK, dV, O, torch.from_numpy(key_len).cuda(), mult, 20, flags)
+        torch.cuda.synchronize()
+        assert ctx.hccs_device_status() == 0
+        want = oracle.attention(Q, K, V, mult, 20, theta, oracle_mode(oracle, flags), threads=8, key_len=key_len)
+        assert_same(O.cpu().numpy(), want, f"ring with key lengths, flags={flags}")
+    mult_wide = (mult.astype(np.int64) * 64).astype(np.int32) // 8         # shift 26: the 64-bit flow
+    O = torch.full(Q.shape, 0x7EADBEEF, dtype=torch.int32, device="cuda")
+    ctx.hccs_attention_fused(dQ, dK, dV, O, mult_wide, 26, 0)
+    torch.cuda.synchronize()
+    assert ctx.hccs_device_status() == 0
+    want = oracle.attention(Q, K, V, mult_wide, 26, theta, 0, threads=8)
+    assert_same(O.cpu().numpy(), want, "ring, shift 26")
+    ctx.close()
+
+
 def test_head_dimension_128_many_tiles_and_wide_shift(hccs, oracle):
     """More tiles than SMs (persistent CTAs take several), and the 64-bit requantisation flow."""
     rng = np.random.default_rng(4100)
@@ -114,7 +159,7 @@ def test_unsupported_shapes_are_refused(hccs):
     import torch
     ctx = hccs.Context(0)
     ctx.hccs_params_upload([(31, 1, 20)] * 2, 1024)
-    for L, d in ((128, 32), (2048, 64), (1040, 64), (640, 128), (128, 96)):
+    for L, d in ((128, 32), (2048, 64), (1040, 64), (1040, 128), (128, 96)):
         q = torch.zeros((1, 2, L, d), dtype=torch.int8, device="cuda")
         o = torch.zeros((1, 2, L, d), dtype=torch.int32, device="cuda")
         with pytest.raises(hccs.HccsError) as ei:
