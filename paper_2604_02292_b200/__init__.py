@@ -8,7 +8,7 @@ import importlib
 from . import workloads  # noqa: F401
 
 __all__ = ["workloads"]
-_SUBMODULES = ("build", "binding", "calibrate_report")
+_SUBMODULES = ("build", "binding")
 
 
 def __getattr__(name):

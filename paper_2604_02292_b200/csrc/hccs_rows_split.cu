@@ -1,6 +1,7 @@
 // Register-resident row kernel for Lk = 32*G*V (G lanes per row, V 32-byte chunks per lane):
 // the powers of two from 32 to 8192 and the multiples of 32 below 4096 whose odd part is 3, 5 or 7
-// (and, with 16-byte chunks or padded lane groups, the other multiples of 16: see launch_shape).  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
+// (and, with 16-byte chunks or padded lane groups, every other multiple of 16 up to 4096 and tensors that
+// are only 16-byte aligned: see launch_shape).  Algorithm 1 of the paper, stage by stage, on 16-bit pairs.
 //
 // Why 16-bit pairs: on sm_100a the byte-wise SIMD min/max intrinsics are emulated (about ten
 // instructions each), while min/max on s16x2 and the three-operand forms max(a+b, c) are single
@@ -249,7 +250,12 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                 stg256(p_row + col, lo);
                 stg256(p_row + col + 16, hi);
             } else {
-                stg256(p_row + col, out);
+                // 16-byte chunks also serve tensors that are only 16-byte aligned: two 16-byte stores
+                uint32_t lo[4], hi[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { lo[k] = out[k]; hi[k] = out[4 + k]; }
+                stg128(p_row + col, lo);
+                stg128(p_row + col + 8, hi);
             }
         }
     } else {
@@ -316,10 +322,12 @@ cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t s
     return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL, CW, PAD>, x, p, a);
 }
 
+// align32: both tensors start on a 32-byte boundary (the 32-byte-chunk shapes need it; the 16-byte-chunk
+// shapes only need 16-byte alignment, which the caller has checked).
 template <bool U16, bool CLB, bool CAUSAL>
-cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st, bool *taken) {
+cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st, bool align32, bool *taken) {
     *taken = true;
-    switch (a.Lk) {
+    if (align32) switch (a.Lk) {
         case 32: return launch_gv<1, 1, U16, CLB, CAUSAL>(x, p, a, st);
         case 64:    // int16 output: two lanes per row (30.7 against 31.3 us for 2^20 rows); uint8: a lane per row
             if constexpr (U16) return launch_gv<2, 1, U16, CLB, CAUSAL>(x, p, a, st);
@@ -364,10 +372,12 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
 #undef HCCS_SPLIT16_G
 #undef HCCS_SPLIT16
         }
-        // every other multiple of 16 up to 4096: eight 16-byte chunks per lane, the smallest power of two
-        // of lanes that covers the row, the excess chunks padded (masked path, also without a mask)
+        // every other multiple of 16 up to 4096 (and every one when the tensors are only 16-byte aligned): eight
+        // 16-byte chunks per lane, the smallest power of two of lanes that covers the row, the excess chunks
+        // padded (masked path, also without a mask)
         const int chunks = a.Lk / 16;
-        if (chunks > 8 && chunks <= 8 * 32) {
+        if (chunks <= 8 * 32) {
+            if (chunks <= 8) return launch_gv<1, 8, U16, CLB, true, 4, true>(x, p, a, st);
             if (chunks <= 16) return launch_gv<2, 8, U16, CLB, true, 4, true>(x, p, a, st);
             if (chunks <= 32) return launch_gv<4, 8, U16, CLB, true, 4, true>(x, p, a, st);
             if (chunks <= 64) return launch_gv<8, 8, U16, CLB, true, 4, true>(x, p, a, st);
@@ -375,7 +385,7 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
             return launch_gv<32, 8, U16, CLB, true, 4, true>(x, p, a, st);
         }
         // ... and the multiples of 32 from there to 8192: eight 32-byte chunks per lane, a whole warp per row
-        if (a.Lk % 32 == 0 && a.Lk <= 8192) return launch_gv<32, 8, U16, CLB, true, 8, true>(x, p, a, st);
+        if (align32 && a.Lk % 32 == 0 && a.Lk <= 8192) return launch_gv<32, 8, U16, CLB, true, 8, true>(x, p, a, st);
     }
     *taken = false;
     return cudaSuccess;
@@ -386,17 +396,18 @@ cudaError_t launch_shape(const int8_t *x, void *p, const RowArgs &a, cudaStream_
 cudaError_t try_launch_split(const int8_t *logits, void *probs, const RowArgs &a, uint32_t flags,
                              cudaStream_t stream, bool *taken) {
     *taken = false;
-    if ((((uintptr_t)logits | (uintptr_t)probs) & 31u) != 0) return cudaSuccess;
+    if ((((uintptr_t)logits | (uintptr_t)probs) & 15u) != 0) return cudaSuccess;
     if (!(flags & 1u) && a.out_shift > 1) return cudaSuccess;
+    const bool align32 = (((uintptr_t)logits | (uintptr_t)probs) & 31u) == 0;
     switch (flags & 7u) {
-        case 0: return launch_shape<false, false, false>(logits, probs, a, stream, taken);
-        case 1: return launch_shape<true, false, false>(logits, probs, a, stream, taken);
-        case 2: return launch_shape<false, true, false>(logits, probs, a, stream, taken);
-        case 3: return launch_shape<true, true, false>(logits, probs, a, stream, taken);
-        case 4: return launch_shape<false, false, true>(logits, probs, a, stream, taken);
-        case 5: return launch_shape<true, false, true>(logits, probs, a, stream, taken);
-        case 6: return launch_shape<false, true, true>(logits, probs, a, stream, taken);
-        default: return launch_shape<true, true, true>(logits, probs, a, stream, taken);
+        case 0: return launch_shape<false, false, false>(logits, probs, a, stream, align32, taken);
+        case 1: return launch_shape<true, false, false>(logits, probs, a, stream, align32, taken);
+        case 2: return launch_shape<false, true, false>(logits, probs, a, stream, align32, taken);
+        case 3: return launch_shape<true, true, false>(logits, probs, a, stream, align32, taken);
+        case 4: return launch_shape<false, false, true>(logits, probs, a, stream, align32, taken);
+        case 5: return launch_shape<true, false, true>(logits, probs, a, stream, align32, taken);
+        case 6: return launch_shape<false, true, true>(logits, probs, a, stream, align32, taken);
+        default: return launch_shape<true, true, true>(logits, probs, a, stream, align32, taken);
     }
 }
 

@@ -2,7 +2,10 @@
 how close the calibrated HCCS is to an fp64 softmax -- next to the uncalibrated, uniformly drawn
 theta of the workload.  Needs a GPU.
 
-    python -m paper_2604_02292_b200.calibrate_report [--alpha 0.0625]
+    python tests/calibration_report.py [--alpha 0.0625]
+
+A report script, kept with the test infrastructure (it holds softmax / KL arithmetic of its own, which has
+no place in the library package).
 
 Per workload: 64 batch entries are the calibration set (as in the paper's Section "Calibration");
 the report is taken on the following 16 entries.  Columns: mean over rows of max_j |p_j/T - sm_j|
@@ -11,8 +14,12 @@ and of KL(sm || q) for the int16 output path, q = row renormalised to one.
 from __future__ import annotations
 
 import argparse
+import os
+import sys
 
 import numpy as np
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 
 
 def _fidelity(p, x, alpha, valid=None):

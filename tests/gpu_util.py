@@ -19,11 +19,12 @@ def oracle_mode(orc, flags):
     return m
 
 
-def forward_np(ctx, x, flags=0, misalign=0, inplace=False):
+def forward_np(ctx, x, flags=0, misalign=0, inplace=False, out_misalign=None):
     """hccs_forward on a numpy int8 [B,H,Lq,Lk] array; returns the numpy result.
 
     The output lives inside a larger byte buffer filled with a canary value, `misalign` bytes off
-    a 256-byte boundary (also applied to the input); bytes around it must come back untouched."""
+    a 256-byte boundary (also applied to the input; `out_misalign` sets the output's offset in bytes on
+    its own); bytes around it must come back untouched."""
     import torch
     import paper_2604_02292_b200 as pkg
     x = np.ascontiguousarray(x, dtype=np.int8)
@@ -44,7 +45,7 @@ def forward_np(ctx, x, flags=0, misalign=0, inplace=False):
         assert (guard[:PAD + misalign] == 0x11).all() and (guard[PAD + misalign + n:] == 0x11).all()
         return out
     obuf = torch.full((n * osz + 2 * PAD,), CANARY, dtype=torch.uint8, device=dev)
-    off = PAD + misalign * osz
+    off = PAD + (misalign * osz if out_misalign is None else out_misalign)
     oview = obuf[off: off + n * osz]
     probs = (oview.view(torch.uint16) if u16 else oview).view(x.shape)
     ctx.hccs_forward(xin, probs, flags)

@@ -16,9 +16,9 @@ def ctx(hccs):
     c.close()
 
 
-def _check(ctx, orc, wl, flags, out_shift=0, misalign=0, inplace=False, threads=8):
+def _check(ctx, orc, wl, flags, out_shift=0, misalign=0, inplace=False, threads=8, out_misalign=None):
     ctx.hccs_params_upload(wl.theta, wl.n_design, out_shift)
-    got = forward_np(ctx, wl.logits, flags, misalign=misalign, inplace=inplace)
+    got = forward_np(ctx, wl.logits, flags, misalign=misalign, inplace=inplace, out_misalign=out_misalign)
     want = orc.forward(wl.logits, wl.theta, oracle_mode(orc, flags), out_shift, threads=threads)
     assert_same(got, want, f"{wl.name} shape={wl.shape} flags={flags} os={out_shift} mis={misalign}")
     assert ctx.hccs_device_status() == 0
@@ -37,7 +37,7 @@ def test_reduced_configs_all_modes(ctx, oracle, hccs, c, batch, flags):
     _check(ctx, oracle, wl, flags)
 
 
-# row lengths around every dispatch boundary: lane-group sizes, two vectors per lane, the
+# row lengths around every dispatch boundary: lane-group sizes, two chunks per lane, the
 # CTA-per-row kernel, ragged tails and lengths that are no multiple of 16
 LENGTHS = [1, 2, 3, 15, 16, 17, 31, 32, 33, 48, 64, 80, 96, 100, 112, 128, 144, 256, 257, 272, 384,
            496, 512, 528, 1000, 1008, 1024, 1040, 2048, 2064, 2304, 4096, 4112, 5000, 8192, 16384, 32752]
@@ -101,6 +101,16 @@ def test_unaligned_pointers(ctx, oracle, hccs, misalign):
         wl = hccs.workloads.make_rows(9, (1, 2, 6, Lk), kind="gauss")
         for flags in (0, 1, 4):
             _check(ctx, oracle, wl, flags, misalign=misalign)
+
+
+@pytest.mark.parametrize("Lk", [16, 32, 48, 64, 96, 128, 160, 272, 512, 1008, 1024, 2048, 3584, 4096])
+def test_sixteen_byte_aligned_tensors(ctx, oracle, hccs, Lk):
+    """Tensors that start on a 16-byte but not on a 32-byte boundary stay in the register-resident kernel
+    (16-byte chunks, padded lane groups), in every mode."""
+    wl = hccs.workloads.make_rows(11000 + Lk, (2, 3, 37, Lk), kind="gauss")
+    for flags in ALL_FLAGS:
+        _check(ctx, oracle, wl, flags, misalign=16, out_misalign=16)
+        _check(ctx, oracle, wl, flags, misalign=32, out_misalign=48)
 
 
 def test_in_place(ctx, oracle, hccs):
