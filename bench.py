@@ -50,13 +50,13 @@ MODE_FLAGS = {"u8div": 0, "u8clb": 2, "u16div": 1, "u16clb": 3}
 # the middle of the rotating-buffer loop without a cache flush in front of them (so that the lines
 # evicted by a launch are counted like in the timed loop); see profiles/.  None: not captured for
 # the kernel as it stands.
-NCU_TRAFFIC_BYTES = {"config2": None, "config3": None, "config4": None, "config5": None}
+NCU_TRAFFIC_BYTES = {"config2": 135.7e6, "config3": 67.3e6, "config4": 401.0e6, "config5": 175.6e6}
 
 # Fused kernel: warp instructions on the integer (ALU) pipe per launch of workload 5, from the ncu
 # capture under profiles/ (sm__inst_executed_pipe_alu).  The pipe issues one warp instruction per
 # two cycles and scheduler (16 lanes per SM sub-partition), so its peak on 148 SMs x 4 schedulers at
 # 1.965 GHz is 148 * 4 * 1.965e9 / 2 warp instructions per second.
-FUSED_ALU_WARP_INSTR = {"config5": None}
+FUSED_ALU_WARP_INSTR = {"config5": 59.4e6}
 ALU_PIPE_PEAK_WARP_INSTR_S = 148 * 4 * 1.965e9 / 2
 
 
@@ -316,6 +316,7 @@ class Timing:
             t = time_regions(launch, stream, steps, self.warmup, prewarm_s, timed_s, barrier=self.barrier)
         self.intervals.append(t["interval"])
         out = region_stats(t["regions_ms"], steps)
+        out["interval"] = t["interval"]
         out["steps"] = steps
         out["host_enqueue_us_per_step"] = t["host_enqueue_us_per_step"]
         out["prewarm_launches"] = t["prewarm_launches"]
@@ -344,6 +345,14 @@ def time_forward(ctx, wl, mode, timing, dev, keep=None):
     st = timing.run(launch, stream)
     st["launches_total"] = ctx.hccs_launch_count() - n0
     st["flags"], st["mode"], st["nbuf"], st["osz"] = flags, mode, nbuf, osz
+    if osz == 1 and not timing.kernel_only:
+        # yardstick: the runtime's device-to-device copy of the same tensor, same buffers, same protocol
+        def copy(i):
+            ps[i % nbuf].view(torch.int8).copy_(xs[i % nbuf], non_blocking=True)
+        st["memcpy_d2d_ms"] = timing.run(copy, stream, prewarm_s=0.2, timed_s=0.2)["ms_per_step"]
+        for i in range(nbuf):              # the copies went into the output buffers: compute them again
+            launch(i)
+        torch.cuda.synchronize()
     if keep is not None:
         keep.update(host_x=host_x, xs=xs, ps=ps, flags=flags, odt=odt, osz=osz, nbuf=nbuf)
     return st, ps[nbuf - 1]
@@ -631,6 +640,8 @@ def run_ours(args):
                 line["e2e"] = e2e
             if osz == 1 and full:
                 line["fidelity"] = fidelity(wl, last_out.cpu().numpy())
+            if "memcpy_d2d_ms" in st:
+                line["timing"]["memcpy_d2d_ms"] = st["memcpy_d2d_ms"]
             if world == 1 and full:
                 cores = os.cpu_count() or 1
                 cpu_rate, cpu_passes, cpu_dt = cpu_oracle_rate(wl, flags, 10.0, cores)
@@ -648,7 +659,7 @@ def run_ours(args):
             for mode in ("u8clb", "u16div", "u16clb"):
                 s2, out2 = time_forward(ctx, wl, mode, timing, dev)
                 r2 = rates(wl, s2)
-                others[f"config2_{mode}"] = leg_summary(wl, s2, r2, full_parity(wl, s2["flags"], out2))
+                others[f"config2_{mode}"] = leg_summary(wl, s2, r2, full_parity(wl, s2["flags"], out2), timing)
                 del out2
                 torch.cuda.empty_cache()
             for c in (3, 4):
@@ -656,14 +667,14 @@ def run_ours(args):
                 ctx.hccs_params_upload(w.theta, w.n_design)
                 s2, out2 = time_forward(ctx, w, "u8div", timing, dev)
                 r2 = rates(w, s2)
-                others[w.name] = leg_summary(w, s2, r2, full_parity(w, s2["flags"], out2))
+                others[w.name] = leg_summary(w, s2, r2, full_parity(w, s2["flags"], out2), timing)
                 others[w.name]["fidelity"] = fidelity(w, out2.cpu().numpy())
                 del out2, w
                 torch.cuda.empty_cache()
             w = workloads.make_config(1)
             ctx.hccs_params_upload(w.theta, w.n_design)
             s2, out2 = time_forward(ctx, w, "u8div", timing, dev)
-            others[w.name] = leg_summary(w, s2, rates(w, s2), full_parity(w, s2["flags"], out2))
+            others[w.name] = leg_summary(w, s2, rates(w, s2), full_parity(w, s2["flags"], out2), timing)
             others[w.name]["note"] = "32 KiB: launch-bound, reported only"
             w5 = workloads.make_config(5)
             f = fused_leg(ctx, w5, timing, with_e2e=False, with_parity=True)
@@ -678,7 +689,7 @@ def run_ours(args):
     if rank == 0 and line is not None:
         sampler.stop()
         if full:
-            clocks = sampler.summary(timing.intervals)
+            clocks = sampler.summary(timing.intervals[:1])       # the headline leg's pre-warm and timed regions
             line["clocks"] = clocks
             if clocks.get("sm_mhz"):
                 line["timing"]["ms_per_step_x_sm_mhz"] = line["ms_per_step"] * clocks["sm_mhz"]
@@ -691,7 +702,23 @@ def run_ours(args):
     ctx.close()
 
 
-def leg_summary(wl, st, r, mismatches):
+def leg_clock(timing, st):
+    """Median SM clock over the samples taken while this leg's launches ran."""
+    time.sleep(0.06)                       # let the sampler deliver the last samples of the interval
+    c = timing.sampler.summary([st["interval"]])
+    return {"sm_mhz": c.get("sm_mhz"), "samples": c.get("samples"), "reasons": c.get("reasons")}
+
+
+def leg_summary(wl, st, r, mismatches, timing=None):
+    out = leg_summary_core(wl, st, r, mismatches)
+    if timing is not None:
+        out["clocks"] = leg_clock(timing, st)
+    if "memcpy_d2d_ms" in st:
+        out["memcpy_d2d_ms"] = st["memcpy_d2d_ms"]
+    return out
+
+
+def leg_summary_core(wl, st, r, mismatches):
     return {"config": config_dict(wl, st["mode"]), "ms_per_step": st["ms_per_step"],
             "ms_per_step_min": st["ms_per_step_min"], "ms_per_step_max": st["ms_per_step_max"],
             "repeats": st["repeats"], "steps": st["steps"], "rows_per_s": r["rows_per_s"],
