@@ -852,12 +852,22 @@ cudaError_t launch_variant(const CUtensorMap &mq, const CUtensorMap &mk, const C
     // resident: Q, two prefetch slots, a slot per K / V block, the panel; ring: Q, four slots, the panel
     const size_t smem = 1024 + (RING ? (1 + kRingSlots) * kTileBytes : 3 * kTileBytes + (size_t)nblk * kTileBytes) + panel;
     auto kernel = fused_attention_kernel<D, CLB, CAUSAL, RING>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // the attribute is raised once per instantiation and device to the largest size a launch can ask for
+    static bool raised[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !raised[dev]) {
+        constexpr size_t kMaxSmem = 1024 + (RING ? (1 + kRingSlots) * kTileBytes : 3 * kTileBytes + (size_t)kMaxBlocks * kTileBytes) +
+                                    (size_t)kTile * kMaxBlocks * kTile;
+        const size_t want = kMaxSmem < 232448 - 8192 ? kMaxSmem : smem;      // (resident d = 128 never asks for more than 512 keys)
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64 && want >= kMaxSmem) raised[dev] = true;
+    }
     const int64_t tiles = (int64_t)a.B * a.H * nblk;
     int sms = 148;
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const unsigned blocks = (unsigned)(tiles < sms ? tiles : sms);      // persistent: one CTA per SM
     kernel<<<blocks, kThreads, smem, st>>>(mq, mk, mv, mo, a, (int)tiles);
     return cudaGetLastError();
