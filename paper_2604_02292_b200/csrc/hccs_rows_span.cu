@@ -34,11 +34,6 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
-__device__ __forceinline__ uint64_t mad_wide(uint32_t a, uint32_t b, uint64_t c) {
-    uint64_t d;
-    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
-    return d;
-}
 __device__ __forceinline__ uint32_t prefix_mask(int nbytes) {        // low nbytes bytes set (0..4, clamped)
     return nbytes >= 4 ? 0xffffffffu : (nbytes <= 0 ? 0u : (1u << (8 * nbytes)) - 1u);
 }
@@ -173,25 +168,25 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
                 }
             }
         } else {
-            const int sh = 1 - a.out_shift;                        // 0 or 1 (checked by the launcher)
-            const uint32_t rp = rho << sh;
+            // the pair arithmetic of the register-resident kernel: X = s * rho' < 2^24 with the coefficients split
+            // at 8 bits, two 32-bit multiply-adds per pair of keys on 16-bit lanes; OUT_SHIFT is 0 or 1 here
+            const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
             const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
-            const uint64_t A = (uint64_t)a1 + ((uint64_t)a1 << 24);
+            const uint32_t ah2 = (a1 >> 8) * 0x00010001u, al2 = (a1 & 255u) * 0x00010001u;
+            const uint32_t bh = b1 >> 8, bl = b1 & 255u;
             int j = sub;
 #pragma unroll
             for (int k = 0; k < kWordsPerLane; ++k, j += G) {
                 if (j >= W) continue;
                 uint32_t q;
                 if (!CLB) {
-                    const uint64_t pe = mad_wide(prmt(e[k], 0, 0x2440u), b1, A);
-                    const uint64_t po = mad_wide(prmt(o[k], 0, 0x2440u), b1, A);
-                    q = prmt((uint32_t)pe, (uint32_t)(pe >> 32), 0x7562u) + prmt((uint32_t)po, (uint32_t)(po >> 32), 0x5726u);
+                    const uint32_t ye = e[k] * bh + ah2 + prmt(e[k] * bl + al2, 0, 0x4341u);
+                    const uint32_t yo = o[k] * bh + ah2 + prmt(o[k] * bl + al2, 0, 0x4341u);
+                    q = prmt(ye, yo, 0x7351u);
                 } else {
-                    const uint32_t x0 = min(a1 + b1 * (e[k] & 0xffffu), 0x00ffffffu);
-                    const uint32_t x1 = min(a1 + b1 * (o[k] & 0xffffu), 0x00ffffffu);
-                    const uint32_t x2 = min(a1 + b1 * (e[k] >> 16), 0x00ffffffu);
-                    const uint32_t x3 = min(a1 + b1 * (o[k] >> 16), 0x00ffffffu);
-                    q = prmt(prmt(x0, x1, 0x0062u), prmt(x2, x3, 0x0062u), 0x5410u);
+                    const uint32_t ye = __viaddmin_u16x2(e[k] * bh + ah2, prmt(e[k] * bl + al2, 0, 0x4341u), 0x7fff7fffu);
+                    const uint32_t yo = __viaddmin_u16x2(o[k] * bh + ah2, prmt(o[k] * bl + al2, 0, 0x4341u), 0x7fff7fffu);
+                    q = prmt(ye >> 7, yo >> 7, 0x6240u);
                 }
                 q &= word_mask(j);
                 const int left = Lk - 4 * j;
