@@ -24,12 +24,10 @@ struct hccs_ctx {
     uint32_t *h_status = nullptr;           // pinned landing place for it
     cudaEvent_t table_copied = nullptr;     // the staging buffers may be rewritten after this
     cudaEvent_t mult_copied = nullptr;
-    cudaStream_t h2d_stream = nullptr;      // hccs_forward_host: input copies
     cudaStream_t d2h_stream = nullptr;      // hccs_forward_host: output copies
     static constexpr int kMaxPieces = 16;
-    cudaEvent_t ev_in[kMaxPieces] = {};
     cudaEvent_t ev_done[kMaxPieces] = {};
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_join = nullptr;
     int32_t last_cuda_error = 0;
     uint64_t launches = 0;
 };
@@ -169,13 +167,10 @@ hccs_status_t hccs_create(hccs_ctx_t **out, int device) {
     if (e == cudaSuccess) e = cudaHostAlloc(&ctx->h_status, sizeof(uint32_t), cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->table_copied, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->mult_copied, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
     for (int i = 0; i < hccs_ctx::kMaxPieces && e == cudaSuccess; ++i) {
-        e = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
+        e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -198,12 +193,9 @@ hccs_status_t hccs_destroy(hccs_ctx_t *ctx) {
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     if (ctx->table_copied) cudaEventDestroy(ctx->table_copied);
     if (ctx->mult_copied) cudaEventDestroy(ctx->mult_copied);
-    if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
     if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
-    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     for (int i = 0; i < hccs_ctx::kMaxPieces; ++i) {
-        if (ctx->ev_in[i]) cudaEventDestroy(ctx->ev_in[i]);
         if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
     }
     (void)cudaGetLastError();
@@ -303,30 +295,22 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const int64_t osz = (flags & HCCS_OUT_U16) ? 2 : 1;
     // Pieces are whole (b, h) slices, so that a piece's first row has query index 0 and its
-    // head is a pure function of the slice index.  Inputs go up on one stream, results come
-    // down on another, kernels run on the caller's stream, chained by events.
+    // head is a pure function of the slice index.  A piece's input copy and its kernel run in order on
+    // the caller's stream (the kernel of one piece delays the next copy by microseconds only); the
+    // results come down on a second stream, piece by piece behind an event, so that the two copy
+    // directions overlap.  One event hand-over per piece: each costs several microseconds of latency.
     const int64_t slices = (int64_t)B * H;
     const int64_t slice_bytes = (int64_t)Lq * Lk;
     int pieces = 1;
     if (slices * slice_bytes >= (8ll << 20)) pieces = 8;
     if (pieces > slices) pieces = (int)slices;
-    HCCS_CUDA(ctx, cudaEventRecord(ctx->ev_fork, stream));
-    HCCS_CUDA(ctx, cudaStreamWaitEvent(ctx->h2d_stream, ctx->ev_fork, 0));
-    HCCS_CUDA(ctx, cudaStreamWaitEvent(ctx->d2h_stream, ctx->ev_fork, 0));
     for (int p = 0; p < pieces; ++p) {
         const int64_t s0 = slices * p / pieces, s1 = slices * (p + 1) / pieces;
         const int64_t off = s0 * slice_bytes, bytes = (s1 - s0) * slice_bytes;
         HCCS_CUDA(ctx, cudaMemcpyAsync(logits_staging + off, logits_host + off, bytes,
-                                       cudaMemcpyHostToDevice, ctx->h2d_stream));
-        HCCS_CUDA(ctx, cudaEventRecord(ctx->ev_in[p], ctx->h2d_stream));
-    }
-    for (int p = 0; p < pieces; ++p) {
-        const int64_t s0 = slices * p / pieces, s1 = slices * (p + 1) / pieces;
-        const int64_t off = s0 * slice_bytes;
-        HCCS_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_in[p], 0));
-        // a piece starts at slice s0: rotate the head index by running the kernel on a view whose
-        // flat row 0 is that slice; (r / Lq) mod H then needs the slice offset folded in, which
-        // the row arguments carry as a starting slice
+                                       cudaMemcpyHostToDevice, stream));
+        // a piece starts at slice s0: the kernel runs on a view whose flat row 0 is that slice, and the
+        // row arguments carry the starting slice so that (r / Lq) mod H still gives the head
         hccs::RowArgs a = make_row_args(ctx, (int32_t)((s1 - s0) * Lq), H, Lq, Lk, flags, nullptr);
         a.slice0 = (int32_t)s0;
         HCCS_CUDA(ctx, hccs::launch_rows(logits_staging + off, (char *)probs_staging + off * osz, a,
@@ -334,8 +318,7 @@ hccs_status_t hccs_forward_host(hccs_ctx_t *ctx, const int8_t *logits_host, void
         HCCS_CUDA(ctx, cudaEventRecord(ctx->ev_done[p], stream));
         HCCS_CUDA(ctx, cudaStreamWaitEvent(ctx->d2h_stream, ctx->ev_done[p], 0));
         HCCS_CUDA(ctx, cudaMemcpyAsync((char *)probs_host + off * osz, (char *)probs_staging + off * osz,
-                                       (s1 - s0) * slice_bytes * osz, cudaMemcpyDeviceToHost,
-                                       ctx->d2h_stream));
+                                       bytes * osz, cudaMemcpyDeviceToHost, ctx->d2h_stream));
     }
     HCCS_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->d2h_stream));
     HCCS_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_join, 0));
