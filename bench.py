@@ -102,10 +102,16 @@ class ClockSampler:
             if len(parts) < 9:
                 continue
             try:
-                t = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
                 sm, mx = float(parts[1]), float(parts[2])
             except ValueError:
                 continue
+            t = time.time()                 # if the tool's own time stamp cannot be read: the time the line arrived
+            for fmt in ("%Y/%m/%d %H:%M:%S.%f", "%Y/%m/%d %H:%M:%S"):
+                try:
+                    t = datetime.datetime.strptime(parts[0], fmt).timestamp()
+                    break
+                except ValueError:
+                    pass
             try:
                 power = float(parts[3])
             except ValueError:
