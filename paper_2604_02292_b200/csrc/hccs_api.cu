@@ -237,7 +237,7 @@ hccs_status_t hccs_params_upload(hccs_ctx_t *ctx, const hccs_head_params_t *para
         e.B = params[h].B;
         e.S = params[h].S;
         e.D = params[h].Dmax;
-        e.Drep = (uint32_t)params[h].Dmax * 0x01010101u;
+        e.pad = 0;
         ctx->h_table[h] = e;
     }
     HCCS_CUDA(ctx, cudaMemcpyAsync(ctx->d_table, ctx->h_table, sizeof(hccs::HeadEntry) * num_heads,

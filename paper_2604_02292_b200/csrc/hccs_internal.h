@@ -11,8 +11,8 @@ namespace hccs {
 struct __align__(16) HeadEntry {
     int32_t B;        // B_h
     int32_t S;        // S_h
-    uint32_t Drep;    // Dmax_h replicated into the four bytes of a word
     int32_t D;        // Dmax_h
+    int32_t pad;      // (keeps the entry at one 16-byte load)
 };
 
 // Division of a 31-bit dividend by a runtime constant: q = (umulhi(n, mul) + n) >> shift.

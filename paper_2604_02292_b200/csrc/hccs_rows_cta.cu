@@ -415,7 +415,7 @@ extern "C" hccs_status_t hccs_forward_static_scratch(const hccs_head_params_t *p
         table.entry[h].B = params[h].B;
         table.entry[h].S = params[h].S;
         table.entry[h].D = params[h].Dmax;
-        table.entry[h].Drep = (uint32_t)params[h].Dmax * 0x01010101u;
+        table.entry[h].pad = 0;
     }
     hccs::HeadEntry *d_table = reinterpret_cast<hccs::HeadEntry *>(scratch + kStaticTableOffsetWords);
     static_scratch_fill_kernel<<<1, 256, 0, stream>>>(scratch, table, num_heads);
