@@ -45,31 +45,44 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+def _declare(L: ctypes.CDLL) -> ctypes.CDLL:
+    """Argument and result types of every function of the C file."""
+    L.hccs_oracle_check_params.argtypes = [_i64] * 4
+    L.hccs_oracle_check_params.restype = ctypes.c_int
+    L.hccs_oracle_rho.argtypes = [_i64, ctypes.c_int]
+    L.hccs_oracle_rho.restype = _i64
+    L.hccs_oracle_row.argtypes = [_p, _p, _i64, _i64, _i64, _i64, ctypes.c_int, _i64,
+                                  _p, _p, _p]
+    L.hccs_oracle_row.restype = _i64
+    L.hccs_oracle_forward.argtypes = [_p, _p, _i64, _i64, _i64, _i64, _p, ctypes.c_int,
+                                      _i64, _i64, _i64, _p, _p, _p]
+    L.hccs_oracle_forward.restype = ctypes.c_int
+    L.hccs_oracle_requant.argtypes = [_i64, _i64, _i64]
+    L.hccs_oracle_requant.restype = _i64
+    L.hccs_oracle_requant_output.argtypes = [_p, _p, _p, _i64, _i64, _i64, _i64, _i64]
+    L.hccs_oracle_requant_output.restype = None
+    L.hccs_oracle_attention.argtypes = [_p, _p, _p, _p, _p, _i64, _p,
+                                        _i64, _i64, _i64, _i64, ctypes.c_int, _i64,
+                                        _i64, _i64, _i64, _i64, _p, _p, _p, _p, _p, _p]
+    L.hccs_oracle_attention.restype = ctypes.c_int
+    return L
+
+
 def lib() -> ctypes.CDLL:
     global _lib
     with _lock:
         if _lib is None:
-            L = ctypes.CDLL(build())
-            L.hccs_oracle_check_params.argtypes = [_i64] * 4
-            L.hccs_oracle_check_params.restype = ctypes.c_int
-            L.hccs_oracle_rho.argtypes = [_i64, ctypes.c_int]
-            L.hccs_oracle_rho.restype = _i64
-            L.hccs_oracle_row.argtypes = [_p, _p, _i64, _i64, _i64, _i64, ctypes.c_int, _i64,
-                                          _p, _p, _p]
-            L.hccs_oracle_row.restype = _i64
-            L.hccs_oracle_forward.argtypes = [_p, _p, _i64, _i64, _i64, _i64, _p, ctypes.c_int,
-                                              _i64, _i64, _i64, _p, _p, _p]
-            L.hccs_oracle_forward.restype = ctypes.c_int
-            L.hccs_oracle_requant.argtypes = [_i64, _i64, _i64]
-            L.hccs_oracle_requant.restype = _i64
-            L.hccs_oracle_requant_output.argtypes = [_p, _p, _p, _i64, _i64, _i64, _i64, _i64]
-            L.hccs_oracle_requant_output.restype = None
-            L.hccs_oracle_attention.argtypes = [_p, _p, _p, _p, _p, _i64, _p,
-                                                _i64, _i64, _i64, _i64, ctypes.c_int, _i64,
-                                                _i64, _i64, _i64, _i64, _p, _p, _p, _p, _p, _p]
-            L.hccs_oracle_attention.restype = ctypes.c_int
-            _lib = L
+            _lib = _declare(ctypes.CDLL(build()))
     return _lib
+
+
+def use_library(path):
+    """Makes every function of this module call the shared library at ``path`` (None: back to the one
+    built from ``hccs_oracle.c``).  For the mutation test only, which plants mistakes in copies of the
+    C file and checks that the pins notice."""
+    global _lib
+    with _lock:
+        _lib = None if path is None else _declare(ctypes.CDLL(path))
 
 
 def _ptr(a):
