@@ -227,9 +227,10 @@ def config_dict(wl, mode):
     flags = int(wl.flags) | MODE_FLAGS[mode]
     osz = 2 if flags & 1 else 1
     n = buffer_sets(wl, osz)
+    total = (1 + osz) * wl.elements * n
+    note = "> L2" if total > L2_BYTES else "fits the L2: a launch-bound workload, not a bandwidth figure"
     return {"workload": wl.name, "shape": list(wl.shape), "flags": flags, "mode": mode,
-            "cache": f"GPU arm: {n} rotating buffer sets ({(1 + osz) * wl.elements * n >> 20} MiB) > L2; "
-                     "CPU arm: the one host copy"}
+            "cache": f"GPU arm: {n} rotating buffer sets ({total >> 20} MiB) {note}; CPU arm: the one host copy"}
 
 
 def algorithmic_bytes(wl, flat: bool):
