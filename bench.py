@@ -385,29 +385,60 @@ def full_parity(wl, flags, got_tensor):
     return int((got_tensor.cpu().numpy() != want).sum())
 
 
-def fidelity(wl, probs_u8, alpha=1.0 / 16, max_rows=4096):
-    """Max-abs error and KL of the kernel's uint8 rows against an fp64 exp-softmax of alpha * x on a
-    seeded row sample (a report, not a gate; theta is uncalibrated)."""
+def fidelity_arrays(logits, probs, flags, T, alpha=1.0 / 16, max_rows=4096):
+    """Max-abs error and KL of integer probability rows (scale T) against an fp64 exp-softmax of alpha * x
+    on a seeded row sample (a report, not a gate)."""
     import numpy as np
-    Bt, H, Lq, Lk = wl.shape
+    Bt, H, Lq, Lk = logits.shape
+    rows = Bt * H * Lq
     rng = np.random.default_rng(0)
-    pick = np.sort(rng.choice(wl.rows, size=min(max_rows, wl.rows), replace=False))
-    x = wl.logits.reshape(-1, Lk)[pick].astype(np.float64)
-    p = probs_u8.reshape(-1, Lk)[pick].astype(np.float64)
+    pick = np.sort(rng.choice(rows, size=min(max_rows, rows), replace=False))
+    x = logits.reshape(-1, Lk)[pick].astype(np.float64)
+    p = probs.reshape(-1, Lk)[pick].astype(np.float64)
     qi = pick % Lq
-    valid = (np.arange(Lk)[None, :] <= qi[:, None] + (Lk - Lq)) if wl.flags & 4 else np.ones(x.shape, bool)
+    valid = (np.arange(Lk)[None, :] <= qi[:, None] + (Lk - Lq)) if flags & 4 else np.ones(x.shape, bool)
     z = np.where(valid, alpha * x, -np.inf)
     z = z - z.max(axis=1, keepdims=True)
     e = np.exp(z)
     sm = e / e.sum(axis=1, keepdims=True)
-    err = np.abs(p / 255.0 - sm).max(axis=1)
+    err = np.abs(p / float(T) - sm).max(axis=1)
     q = np.where(valid, np.maximum(p, 1e-12), 0.0)
     q = q / q.sum(axis=1, keepdims=True)
     with np.errstate(divide="ignore", invalid="ignore"):
         kl = np.where(sm > 0, sm * (np.log(sm) - np.log(np.where(q > 0, q, 1.0))), 0.0).sum(axis=1)
     return {"alpha": alpha, "rows": int(pick.size), "mean_max_abs": float(err.mean()),
-            "worst_max_abs": float(err.max()), "mean_kl": float(kl.mean()),
-            "note": "uint8 output / 255 against fp64 softmax(alpha x); theta uniform in the band, uncalibrated"}
+            "worst_max_abs": float(err.max()), "mean_kl": float(kl.mean())}
+
+
+def fidelity(wl, probs_u8, alpha=1.0 / 16, max_rows=4096):
+    """The kernel's uint8 rows of a whole workload against fp64 softmax(alpha x); theta is uncalibrated."""
+    out = fidelity_arrays(wl.logits, probs_u8, wl.flags, 255, alpha, max_rows)
+    out["note"] = "uint8 output / 255 against fp64 softmax(alpha x); theta uniform in the band, uncalibrated"
+    return out
+
+
+def calibrated_fidelity(ctx, wl, dev, alpha=1.0 / 16):
+    """The paper's offline calibration on synthetic logits: theta per head by the grid scan (hccs_calibrate)
+    on the first 64 batch entries, fidelity of the int16 path on the next 64 with the workload's
+    uniformly drawn theta and with the calibrated one."""
+    import torch
+    import paper_2604_02292_b200 as pkg
+    x = torch.from_numpy(wl.logits[:128]).to(dev)
+    t0 = time.perf_counter()
+    theta_cal, kl_cal = pkg.hccs_calibrate(x[:64].contiguous(), alpha, (2, 127, 1, 0, 127, 1, 1))
+    dt = time.perf_counter() - t0
+    out = {"alpha": alpha, "calibration_set": "batch entries 0..63", "held_out": "batch entries 64..127",
+           "grid": "Dmax 2..127, S 0..127, every B of the band", "calibration_s": dt,
+           "theta_calibrated": theta_cal.tolist(), "objective_on_calibration_set": [float(v) for v in kl_cal]}
+    held = x[64:].contiguous()
+    for name, theta in (("uniform_in_band", wl.theta), ("calibrated", theta_cal)):
+        ctx.hccs_params_upload(theta, wl.n_design)
+        p = torch.empty(held.shape, dtype=torch.uint16, device=dev)
+        ctx.hccs_forward(held, p, int(wl.flags) | 1)
+        torch.cuda.synchronize()
+        out[name] = fidelity_arrays(wl.logits[64:128], p.cpu().numpy(), wl.flags, 32767, alpha)
+    ctx.hccs_params_upload(wl.theta, wl.n_design)
+    return out
 
 
 def fused_leg(ctx, wl, timing, with_e2e, with_parity):
@@ -663,6 +694,7 @@ def run_ours(args):
         # ---------------- the other workloads and modes, same protocol, same line
         if extras and rank == 0:
             others = {}
+            line["fidelity_calibrated_int16"] = calibrated_fidelity(ctx, wl, dev)
             for mode in ("u8clb", "u16div", "u16clb"):
                 s2, out2 = time_forward(ctx, wl, mode, timing, dev)
                 r2 = rates(wl, s2)
