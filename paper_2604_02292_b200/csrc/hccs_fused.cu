@@ -674,10 +674,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                             const uint32_t yo = ro * b1h + ah2 + prmt(ro * b1l + al2, 0, 0x4341u);
                             q = prmt(ye, yo, 0x7351u);
                         } else {
-                            // saturation at 255 folded into the add: Y stops at 255*128 + 127, p = Y >> 7
+                            // saturation at 255 folded into the add: Y stops at 255*128 + 127, p = Y >> 7 = high byte of 2*Y
                             const uint32_t ye = __viaddmin_u16x2(re * b1h + ah2, prmt(re * b1l + al2, 0, 0x4341u), 0x7fff7fffu);
                             const uint32_t yo = __viaddmin_u16x2(ro * b1h + ah2, prmt(ro * b1l + al2, 0, 0x4341u), 0x7fff7fffu);
-                            q = prmt(ye >> 7, yo >> 7, 0x6240u);
+                            q = prmt(ye * 2u, yo * 2u, 0x7351u);
                         }
                         if (CAUSAL) {
                             const int nb = nv - (kb * kTile + (2 * grp + c) * 16 + 4 * k);

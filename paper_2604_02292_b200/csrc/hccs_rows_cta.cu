@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kThreads) rows_cta_kernel(const int8_t *x_all,
                         } else {
                             const uint32_t ye = __viaddmin_u16x2(ev * bh + ah2, prmt(ev * bl + al2, 0, 0x4341u), 0x7fff7fffu);
                             const uint32_t yo = __viaddmin_u16x2(od * bh + ah2, prmt(od * bl + al2, 0, 0x4341u), 0x7fff7fffu);
-                            q = prmt(ye >> 7, yo >> 7, 0x6240u);
+                            q = prmt(ye * 2u, yo * 2u, 0x7351u);
                         }
                         if (CAUSAL) q &= byte_prefix_mask(j.nv - 16 * v - 4 * k);
                         o[k] = q;

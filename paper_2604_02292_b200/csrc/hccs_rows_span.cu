@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
                 } else {
                     const uint32_t ye = __viaddmin_u16x2(e[k] * bh + ah2, prmt(e[k] * bl + al2, 0, 0x4341u), 0x7fff7fffu);
                     const uint32_t yo = __viaddmin_u16x2(o[k] * bh + ah2, prmt(o[k] * bl + al2, 0, 0x4341u), 0x7fff7fffu);
-                    q = prmt(ye >> 7, yo >> 7, 0x6240u);
+                    q = prmt(ye * 2u, yo * 2u, 0x7351u);
                 }
                 q &= word_mask(j);
                 const int left = Lk - 4 * j;

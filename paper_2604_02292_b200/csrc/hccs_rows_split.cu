@@ -289,10 +289,10 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                         out[k] = prmt(ye, yo, 0x7351u);
                     } else {
                         // the leading-bit reciprocal can overshoot: Y saturates at 255*128 + 127 in the add
-                        // itself, and p = Y >> 7 is then bits 7..14 of each lane (bytes 0 and 2 after the shift)
+                        // itself, and p = Y >> 7 is the high byte of each lane of 2*Y (the doubling runs on the multiply pipe)
                         const uint32_t ye = __viaddmin_u16x2(re * bh + ah2, prmt(re * bl + al2, 0, 0x4341u), 0x7fff7fffu);
                         const uint32_t yo = __viaddmin_u16x2(ro * bh + ah2, prmt(ro * bl + al2, 0, 0x4341u), 0x7fff7fffu);
-                        out[k] = prmt(ye >> 7, yo >> 7, 0x6240u);
+                        out[k] = prmt(ye * 2u, yo * 2u, 0x7351u);
                     }
                 }
                 if (!full[v]) {
