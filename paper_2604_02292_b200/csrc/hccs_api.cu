@@ -351,7 +351,7 @@ static hccs_status_t fused_common(hccs_ctx_t *ctx, const int8_t *Q, const int8_t
     if (L > ctx->n_design) return HCCS_ERR_CONSTRAINT;
     if ((int64_t)B * H * L * d == 0) return HCCS_OK;
     if (!Q || !K || !V || !O) return HCCS_ERR_INVALID_ARG;
-    if (!hccs::fused_shape_supported(L, d) || ctx->out_shift > 1) return HCCS_ERR_UNSUPPORTED;
+    if (!hccs::fused_shape_supported(L, d)) return HCCS_ERR_UNSUPPORTED;
     if ((((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O) & 15u) != 0)
         return HCCS_ERR_UNSUPPORTED;
     DeviceGuard g(ctx->device);

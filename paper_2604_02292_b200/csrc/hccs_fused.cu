@@ -650,7 +650,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // b1 = b1h*256 + b1l, X >> 8 = ah + b1h*r + ((al + b1l*r) >> 8) < 2^16, and every partial result fits
             // its lane (r <= 127).  (A 64-bit multiply-add with the keys 24 bits apart needs one multiply per
             // pair instead of two, but its 64-bit addend costs two more instructions on the integer pipe.)
-            const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
+            // (an OUT_SHIFT above 1 is computed as OUT_SHIFT = 1 and the packed bytes are shifted by the rest)
+            const int eff_shift = min(a.out_shift, 1), post_shift = a.out_shift - eff_shift;
+            const uint32_t post_mask = (0xffu >> post_shift) * 0x01010101u;
+            const uint32_t rp = CLB ? (rho >> eff_shift) : (rho << (1 - eff_shift));
             const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
             const uint32_t ah2 = (a1 >> 8) * 0x00010001u, al2 = (a1 & 255u) * 0x00010001u;
             const uint32_t b1h = b1 >> 8, b1l = b1 & 255u;
@@ -679,6 +682,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                             const uint32_t yo = __viaddmin_u16x2(ro * b1h + ah2, prmt(ro * b1l + al2, 0, 0x4341u), 0x7fff7fffu);
                             q = prmt(ye * 2u, yo * 2u, 0x7351u);
                         }
+                        if (post_shift) q = (q >> post_shift) & post_mask;
                         if (CAUSAL) {
                             const int nb = nv - (kb * kTile + (2 * grp + c) * 16 + 4 * k);
                             q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);

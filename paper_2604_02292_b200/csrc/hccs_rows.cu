@@ -3,15 +3,14 @@
 // Four kernels, all integer-only and bit-exact by construction (integer max and sum are
 // order-independent, so any reduction tree gives the one correct result).  launch_mode picks, in this order:
 //   rows_split_kernel    (hccs_rows_split.cu) Lk % 16 == 0 up to 4096 (and the multiples of 32 up to 8192),
-//                        16-byte aligned tensors, OUT_SHIFT <= 1: rows held in registers by groups of
-//                        lanes, 32- or 16-byte chunks; the fast path.
-//   rows_span_kernel     (hccs_rows_span.cu) any other Lk up to 1024 and any alignment, OUT_SHIFT <= 1: runs
-//                        of rows moved through shared memory as contiguous spans.
-//   rows_cta_kernel      (hccs_rows_cta.cu) longer rows with Lk % 16 == 0 and 16-byte aligned tensors, any
-//                        OUT_SHIFT: one CTA per row, the row staged in shared memory by bulk asynchronous
-//                        copies (TMA).
-//   rows_generic_kernel  (this file) everything else (any Lk, any alignment, any OUT_SHIFT): one warp per
-//                        row, byte accesses.
+//                        16-byte aligned tensors: rows held in registers by groups of lanes, 32- or 16-byte
+//                        chunks; the fast path.
+//   rows_span_kernel     (hccs_rows_span.cu) any other Lk up to 1024 and any alignment: runs of rows moved
+//                        through shared memory as contiguous spans.
+//   rows_cta_kernel      (hccs_rows_cta.cu) longer rows with Lk % 16 == 0 and 16-byte aligned tensors: one CTA
+//                        per row, the row staged in shared memory by bulk asynchronous copies (TMA).
+//   rows_generic_kernel  (this file) everything else (any Lk, any alignment): one warp per row, byte accesses.
+// Every kernel takes every OUT_SHIFT of the int8 output path.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -81,14 +80,13 @@ cudaError_t launch_generic(const int8_t *x, void *p, const RowArgs &a, cudaStrea
 template <bool U16, bool CLB, bool CAUSAL>
 cudaError_t launch_mode(const int8_t *x, void *p, const RowArgs &a, cudaStream_t st) {
     const bool aligned = (((uintptr_t)x | (uintptr_t)p) & 15u) == 0 && a.Lk % 16 == 0;
-    const bool shift_ok = U16 || a.out_shift <= 1;
-    if (aligned && shift_ok) {
+    if (aligned) {
         bool taken = false;
         cudaError_t e = try_launch_split(x, p, a, (U16 ? 1u : 0u) | (CLB ? 2u : 0u) | (CAUSAL ? 4u : 0u), st,
                                          &taken);
         if (taken) return e;
     }
-    if (shift_ok && a.Lk <= 1024) {         // any other length or alignment: rows moved as contiguous spans
+    if (a.Lk <= 1024) {                     // any other length or alignment: rows moved as contiguous spans
         bool taken = false;
         cudaError_t e = try_launch_span(x, p, a, (U16 ? 1u : 0u) | (CLB ? 2u : 0u) | (CAUSAL ? 4u : 0u), st, &taken);
         if (taken) return e;

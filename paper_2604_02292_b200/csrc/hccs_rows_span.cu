@@ -169,8 +169,11 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
             }
         } else {
             // the pair arithmetic of the register-resident kernel: X = s * rho' < 2^24 with the coefficients split
-            // at 8 bits, two 32-bit multiply-adds per pair of keys on 16-bit lanes; OUT_SHIFT is 0 or 1 here
-            const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
+            // at 8 bits, two 32-bit multiply-adds per pair of keys on 16-bit lanes
+            // an OUT_SHIFT above 1 is computed as OUT_SHIFT = 1 and the packed bytes are shifted by the rest
+            const int eff_shift = min(a.out_shift, 1), post_shift = a.out_shift - eff_shift;
+            const uint32_t post_mask = (0xffu >> post_shift) * 0x01010101u;
+            const uint32_t rp = CLB ? (rho >> eff_shift) : (rho << (1 - eff_shift));
             const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
             const uint32_t ah2 = (a1 >> 8) * 0x00010001u, al2 = (a1 & 255u) * 0x00010001u;
             const uint32_t bh = b1 >> 8, bl = b1 & 255u;
@@ -188,6 +191,7 @@ __global__ void __launch_bounds__(kSpanThreads) rows_span_kernel(const int8_t *x
                     const uint32_t yo = __viaddmin_u16x2(o[k] * bh + ah2, prmt(o[k] * bl + al2, 0, 0x4341u), 0x7fff7fffu);
                     q = prmt(ye * 2u, yo * 2u, 0x7351u);
                 }
+                if (post_shift) q = (q >> post_shift) & post_mask;
                 q &= word_mask(j);
                 const int left = Lk - 4 * j;
                 uint8_t *dst = smem + ob + 4 * j;
@@ -247,7 +251,6 @@ cudaError_t try_launch_span(const int8_t *logits, void *probs, const RowArgs &a,
                             cudaStream_t stream, bool *taken) {
     *taken = false;
     if (a.Lk < 1 || a.Lk > 4 * kMaxWordsPerLane * 32) return cudaSuccess;  // 1024 keys at most
-    if (!(flags & 1u) && a.out_shift > 1) return cudaSuccess;
     *taken = true;
     switch (flags & 7u) {
         case 0: return launch_span<false, false, false>(logits, probs, a, stream);

@@ -261,8 +261,12 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     } else {
         // rho' = rho << (1 - OUT_SHIFT) and p = X >> 16 for the divide; rho' = rho >> OUT_SHIFT (exact: the
         // leading-bit rho is 255 * 2^(15-k), k <= 14) and p = min(X >> 15, 255) for the leading-bit form, so
-        // that X = s * rho' stays below 2^24 in both (s <= Z < 2^(k+1)); OUT_SHIFT is 0 or 1 (the launcher checks)
-        const uint32_t rp = CLB ? (rho >> a.out_shift) : (rho << (1 - a.out_shift));
+        // that X = s * rho' stays below 2^24 in both (s <= Z < 2^(k+1)).  That covers OUT_SHIFT 0 and 1; a
+        // larger OUT_SHIFT is computed as OUT_SHIFT = 1 (no result above 127 / 255, no saturation) and the
+        // packed bytes are shifted right by the rest afterwards: floor(floor(a / b) / c) = floor(a / (b c)).
+        const int eff_shift = min(a.out_shift, 1), post_shift = a.out_shift - eff_shift;
+        const uint32_t post_mask = (0xffu >> post_shift) * 0x01010101u;
+        const uint32_t rp = CLB ? (rho >> eff_shift) : (rho << (1 - eff_shift));
         const uint32_t a1 = (uint32_t)F * rp, b1 = (uint32_t)th.S * rp;
         // X = a1 + b1*r.  With a1 = ah*256 + al and
         // b1 = bh*256 + bl, X >> 8 = ah + bh*r + ((al + bl*r) >> 8) =: Y < 2^16, and both ah + bh*r and
@@ -294,6 +298,10 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
                         const uint32_t yo = __viaddmin_u16x2(ro * bh + ah2, prmt(ro * bl + al2, 0, 0x4341u), 0x7fff7fffu);
                         out[k] = prmt(ye * 2u, yo * 2u, 0x7351u);
                     }
+                }
+                if (post_shift) {                              // uniform: OUT_SHIFT >= 2
+#pragma unroll
+                    for (int k = 0; k < CW; ++k) out[k] = (out[k] >> post_shift) & post_mask;
                 }
                 if (!full[v]) {
 #pragma unroll
@@ -397,7 +405,6 @@ cudaError_t try_launch_split(const int8_t *logits, void *probs, const RowArgs &a
                              cudaStream_t stream, bool *taken) {
     *taken = false;
     if ((((uintptr_t)logits | (uintptr_t)probs) & 15u) != 0) return cudaSuccess;
-    if (!(flags & 1u) && a.out_shift > 1) return cudaSuccess;
     const bool align32 = (((uintptr_t)logits | (uintptr_t)probs) & 31u) == 0;
     switch (flags & 7u) {
         case 0: return launch_shape<false, false, false>(logits, probs, a, stream, align32, taken);

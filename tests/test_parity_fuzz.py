@@ -23,7 +23,7 @@ def test_random_forward_calls(hccs, oracle, seed):
     while Bt * H * Lq * Lk > (1 << 22):
         Lq = max(1, Lq // 2)
     flags = int(rng.integers(0, 8))
-    out_shift = int(rng.choice([0, 0, 0, 1, 2]))
+    out_shift = int(rng.choice([0, 0, 0, 1, 2, 3, 6]))
     n_design = Lk if rng.random() < 0.6 else int(min(32767, Lk + rng.integers(1, 200)))
     kind = str(rng.choice(["gauss", "laplace", "uniform", "extreme", "const"]))
     wl = hccs.workloads.make_rows(91_000 + seed, (Bt, H, Lq, Lk), n_design=n_design, kind=kind)
@@ -61,7 +61,7 @@ def test_random_fused_calls(hccs, oracle, seed):
     Bt = int(rng.integers(1, 4))
     flags = int(rng.choice([0, 2, 4, 6]))
     sh = int(rng.choice([12, 20, 20, 24, 26]))
-    out_shift = int(rng.choice([0, 0, 1]))
+    out_shift = int(rng.choice([0, 0, 1, 2, 4]))
     lo, hi = (-128, 128) if rng.random() < 0.5 else (-64, 64)
     Q, K, V = (rng.integers(lo, hi, size=(Bt, H, L, d), dtype=np.int8) for _ in range(3))
     theta = hccs.workloads.sample_theta(rng, H, 1024)

@@ -87,9 +87,9 @@ def test_shorter_rows_than_designed(ctx, oracle, hccs):
             _check(ctx, oracle, wl, flags)
 
 
-@pytest.mark.parametrize("out_shift", [0, 1, 2, 5])
+@pytest.mark.parametrize("out_shift", [0, 1, 2, 3, 5, 8])
 def test_out_shift(ctx, oracle, hccs, out_shift):
-    for Lk in (64, 100, 2048):
+    for Lk in (16, 64, 100, 128, 272, 2048, 4112):
         wl = hccs.workloads.make_rows(3, (2, 3, 8, Lk), kind="gauss")
         for flags in (0, 2, 4):
             _check(ctx, oracle, wl, flags, out_shift=out_shift)
