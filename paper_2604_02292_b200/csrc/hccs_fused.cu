@@ -682,12 +682,15 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                             const uint32_t yo = __viaddmin_u16x2(ro * b1h + ah2, prmt(ro * b1l + al2, 0, 0x4341u), 0x7fff7fffu);
                             q = prmt(ye * 2u, yo * 2u, 0x7351u);
                         }
-                        if (post_shift) q = (q >> post_shift) & post_mask;
                         if (CAUSAL) {
                             const int nb = nv - (kb * kTile + (2 * grp + c) * 16 + 4 * k);
                             q &= nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : (1u << (8 * nb)) - 1u);
                         }
                         o[k] = q;
+                    }
+                    if (post_shift) {                              // uniform: OUT_SHIFT >= 2 (masked bytes stay zero)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) o[k] = (o[k] >> post_shift) & post_mask;
                     }
                     *reinterpret_cast<uint4 *>(blk + (((2 * grp + c) ^ swz) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }

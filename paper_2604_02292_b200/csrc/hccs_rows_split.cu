@@ -110,7 +110,7 @@ __device__ __forceinline__ uint32_t byte_mask(int cnt, int k) {
 // no row of the warp reaches it (then it is skipped and stored as zeros), or neither (masked code).  With
 // a causal mask the diagonal crosses exactly one chunk index of a warp, so one chunk per warp pays for masks.
 template <int G, int V, bool U16, bool CLB, bool CAUSAL, int CW = 8, bool PAD = false>
-__global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, void *p_all, RowArgs a, int prefetch_ctas) {
+__global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, void *p_all, RowArgs a) {
     static_assert(!PAD || CAUSAL, "padded lane groups run through the masked path");
     constexpr int RW = 32 / G;      // rows per warp
     constexpr int NW = CW * V;      // 32-bit words of logits per lane
@@ -128,21 +128,16 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     // Programmatic dependent launch: everything above touches no global memory, so it may run
     // while the previous kernel in the stream drains; all reads and writes come after the wait.
     asm volatile("griddepcontrol.launch_dependents;");
-    // While the previous kernel of the stream drains: one bulk prefetch of the warp's tile (its RW rows are
-    // contiguous) into L2, by the CTAs the launcher names (the first `prefetch_ctas` of the grid).  A prefetch is
-    // safe whatever that kernel still writes, because L2 is the point of coherence; the loads behind the wait
-    // then find their lines on the chip.  In a launch of a few waves every CTA does it (3 to 7 % on 128-key causal
-    // heads: the request also leaves a prologue earlier than the lanes' own loads), in a longer one the first
-    // wave only (1 % on 512-key rows; with every CTA prefetching such a launch gets slower).  Not for the
-    // lane-per-row shapes: measured no gain or a loss there (their loads mark the lines evict-first, a prefetched
-    // line keeps its normal priority and crowds the output out of L2).
-    if (G > 1 && (int)blockIdx.x < prefetch_ctas && lane == 0) {
-        const uint32_t row0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RW;
-        if (row0 < (uint32_t)a.rows) {
-            const uint32_t bytes = min((uint32_t)RW, (uint32_t)a.rows - row0) * (uint32_t)a.Lk;   // a multiple of 16
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(x_all + (int64_t)row0 * a.Lk), "r"(bytes)
-                         : "memory");
-        }
+    // Before the wait: one bulk prefetch of the CTA's rows (they are contiguous) into L2.  A prefetch is safe
+    // whatever the previous kernel of the stream still writes, because L2 is the point of coherence; in the first
+    // wave it runs while that kernel drains, and in every wave the request leaves a prologue earlier than the
+    // lanes' own loads: 4 to 7 % on 128-key causal heads, 1 % on 512-key rows.  Not for the lane-per-row shapes:
+    // measured no gain or a loss there (their loads mark the lines evict-first, a prefetched line keeps its normal
+    // priority and crowds the output out of L2).
+    if (G > 1 && threadIdx.x == 0) {
+        const uint32_t cta_row0 = blockIdx.x * (blockDim.x >> 5) * RW;        // (they are contiguous; row0 < rows)
+        const uint32_t bytes = min((blockDim.x >> 5) * RW, (uint32_t)a.rows - cta_row0) * (uint32_t)a.Lk;   // a multiple of 16
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(x_all + (int64_t)cta_row0 * a.Lk), "r"(bytes));
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const HeadEntry th = a.table[head];
@@ -343,11 +338,7 @@ cudaError_t launch_gv(const int8_t *x, void *p, const RowArgs &a, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    // CTAs that prefetch their tiles into L2 before the dependency wait (see the kernel): all of them in a launch
-    // of up to four waves of five CTAs per SM, the first wave in a longer one
-    constexpr unsigned kWave = 5u * 148u;
-    const int prefetch_ctas = G > 1 ? (int)(blocks <= 4u * kWave ? blocks : kWave) : 0;
-    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL, CW, PAD>, x, p, a, prefetch_ctas);
+    return cudaLaunchKernelEx(&cfg, rows_split_kernel<G, V, U16, CLB, CAUSAL, CW, PAD>, x, p, a);
 }
 
 // align32: both tensors start on a 32-byte boundary (the 32-byte-chunk shapes need it; the 16-byte-chunk
