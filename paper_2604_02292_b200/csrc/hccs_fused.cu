@@ -242,17 +242,18 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 
     // Key blocks a tile goes through: all of the head's, or only those that hold a valid key for some row
     // of the tile (causal rule, per-batch key length); at least one, so that O is written.
-    auto blocks_of = [&](int tile) -> int {
+    auto blocks_at = [&](int qt_, int batch_) -> int {      // query tile qt_ of a head of batch entry batch_
         int n = nblk;
         if (CAUSAL) {
-            if (causal) n = tile % nblk + 1;
+            if (causal) n = qt_ + 1;
             if (a.key_len) {
-                const int kl = min(max(a.key_len[tile / nblk / a.H], 0), a.L);
+                const int kl = min(max(a.key_len[batch_], 0), a.L);
                 n = min(n, max((kl + kTile - 1) / kTile, 1));
             }
         }
         return n;
     };
+    auto blocks_of = [&](int tile) -> int { return CAUSAL ? blocks_at(tile % nblk, tile / nblk / a.H) : nblk; };
     // A CTA walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every mbarrier completes
     // one phase per use, so both sides count their uses (per barrier, because a causal tile uses
     // only its first qt + 1 key blocks) and wait on the parity of that count.
@@ -459,6 +460,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             tcgen05_fence_after();
             uint32_t acc[32];
             tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+            tcgen05_fence_before();                      // the accumulators are in registers: the buffer goes back now
+            mbar_arrive(smem_u32(&bars.s_free[sb]));
             const int c0 = kb * kTile + grp * 32;
             if (CAUSAL && c0 + 32 > nv_row) {
 #pragma unroll
@@ -467,33 +470,61 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             }
 #pragma unroll
             for (int e = 0; e < 32; e += 2) amax = __vimax3_s32(amax, (int)acc[e], (int)acc[e + 1]);
-            tcgen05_fence_before();
-            mbar_arrive(smem_u32(&bars.s_free[sb]));
         };
         int amax_carry = -(1 << 30), r1_carry = 0;           // first-round blocks of a tile taken ahead of it
-        // number of valid keys (always a prefix) of this thread's row in the tile of head slice bh_ that
+        // number of valid keys (always a prefix) of this thread's row in a tile of batch entry batch_ that
         // starts at query q0_
-        auto valid_keys = [&](int bh_, int q0_) -> int {
+        auto valid_keys = [&](int batch_, int q0_) -> int {
             int n = a.L;
             if (CAUSAL) {
                 if (causal) n = min(q0_ + t + 1, n);
-                if (a.key_len) n = min(n, max(a.key_len[bh_ / a.H], 0));
+                if (a.key_len) n = min(n, max(a.key_len[batch_], 0));
             }
             return n;
         };
+        // Where a tile is and the constants of its head.  Both are kept one tile ahead: the position advances
+        // by additions (no division per tile), and the head's constants are loaded while the previous tile is
+        // in its last phases -- at the top of a tile their latency (a trip to L2 behind two divisions) stood
+        // in front of every row warp at once.
+        struct TileAt { int bh, qt, head, batch; };
+        struct HeadConsts { int4 th, rq, rx; };   // {B, S, D, -}, {M << k, C << k, -lo, hi - lo}, {out scale, out multiplier, 1/M (double)}
+        const int step_qt = (int)gridDim.x % nblk, step_bh = (int)gridDim.x / nblk;
+        const int step_head = step_bh % a.H, step_batch = step_bh / a.H;
+        auto advance = [&](TileAt p) -> TileAt {
+            p.qt += step_qt;
+            const int carry = p.qt >= nblk ? 1 : 0;
+            p.qt -= carry ? nblk : 0;
+            p.bh += step_bh + carry;
+            p.head += step_head + carry;
+            p.batch += step_batch;
+            if (p.head >= a.H) { p.head -= a.H; ++p.batch; }
+            return p;
+        };
+        auto load_consts = [&](int head_) -> HeadConsts {
+            HeadConsts c;
+            c.th = *reinterpret_cast<const int4 *>(a.table + head_);
+            c.rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head_);       // host-prepared constants
+            c.rx = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head_ + 4);
+            return c;
+        };
+        TileAt cur;
+        cur.bh = (int)blockIdx.x / nblk; cur.qt = (int)blockIdx.x % nblk;
+        cur.head = cur.bh % a.H; cur.batch = cur.bh / a.H;
+        HeadConsts cc = load_consts(cur.head);
 
         for (int tile = blockIdx.x, it = 0; tile < num_tiles; tile += gridDim.x, ++it) {
-            const int bh = tile / nblk, qt = tile % nblk;
-            const int head = bh % a.H;
+            const int bh = cur.bh, qt = cur.qt;
             const int q0 = qt * kTile;
-            const int kblocks = blocks_of(tile);
-            const HeadEntry th = a.table[head];
-            const int4 rq = *reinterpret_cast<const int4 *>(a.requant_mult + 8 * head);   // host-prepared constants
-            const float out_scale = __int_as_float(a.requant_mult[8 * head + 4]);
-            const double inv_m = *reinterpret_cast<const double *>(a.requant_mult + 8 * head + 6);   // 1 / M_h
+            const int kblocks = blocks_at(qt, cur.batch);
+            HeadEntry th;
+            th.B = cc.th.x; th.S = cc.th.y; th.D = cc.th.z;
+            const int4 rq = cc.rq;
+            const float out_scale = __int_as_float(cc.rx.x);
+            const int32_t out_mult = cc.rx.y;
+            const double inv_m = __hiloint2double(cc.rx.w, cc.rx.z);                     // 1 / M_h
             // valid keys of this row: all L of them, the causal prefix, the batch entry's key length
             // (keys at and beyond L exist only as padding of the last block when L is no multiple of 128)
-            const int nv = valid_keys(bh, q0);
+            const int nv = valid_keys(cur.batch, q0);
 
             // the previous tile's O rows were staged in the panel: their bulk copies must have
             // read them before the panel is written again
@@ -562,6 +593,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     uint8_t *blk = row_base + kb * kPanelBlockBytes;
                     uint32_t acc[32];
                     tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+                    tcgen05_fence_before();
+                    mbar_arrive(smem_u32(&bars.s_free[sb]));
                     uint32_t w[8];
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
@@ -576,8 +609,6 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     }
                     *reinterpret_cast<uint4 *>(blk + (((2 * grp) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     *reinterpret_cast<uint4 *>(blk + (((2 * grp + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-                    tcgen05_fence_before();
-                    mbar_arrive(smem_u32(&bars.s_free[sb]));
                 }
             } else {
                 const int32_t mult_hi = rq.x << (32 - a.requant_shift);   // x = high word of acc*mult_hi + 2^31
@@ -590,6 +621,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     uint8_t *blk = row_base + kb * kPanelBlockBytes;
                     uint32_t acc[32];
                     tmem_ld32(tmem + lane_addr + sb * 128 + grp * 32, acc);
+                    tcgen05_fence_before();
+                    mbar_arrive(smem_u32(&bars.s_free[sb]));
                     uint32_t w[8];
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
@@ -604,8 +637,6 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     }
                     *reinterpret_cast<uint4 *>(blk + (((2 * grp) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     *reinterpret_cast<uint4 *>(blk + (((2 * grp + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-                    tcgen05_fence_before();
-                    mbar_arrive(smem_u32(&bars.s_free[sb]));
                 }
                 xmax = min(max(xmax, -128), 127);                     // the stored logits are clamped
                 part_max[grp][t] = xmax;
@@ -704,11 +735,15 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // produced meanwhile (the other K tiles can only be fetched once V is no longer needed)
             amax_carry = -(1 << 30);
             r1_carry = 0;
-            if (two_rounds && tile + (int)gridDim.x < num_tiles) {
-                const int qt_n = (tile + (int)gridDim.x) % nblk;
-                const int kblocks_n = blocks_of(tile + (int)gridDim.x);
-                const int nv_n = valid_keys((tile + (int)gridDim.x) / nblk, qt_n * kTile);
-                for (; ok && r1_carry < min(2, kblocks_n); ++r1_carry) first_round_block(r1_carry, nv_n, amax_carry);
+            const TileAt nxt = advance(cur);
+            HeadConsts nc = cc;
+            if (tile + (int)gridDim.x < num_tiles) {
+                nc = load_consts(nxt.head);                    // used after the next tile's first round
+                if (two_rounds) {
+                    const int kblocks_n = blocks_at(nxt.qt, nxt.batch);
+                    const int nv_n = valid_keys(nxt.batch, nxt.qt * kTile);
+                    for (; ok && r1_carry < min(2, kblocks_n); ++r1_carry) first_round_block(r1_carry, nv_n, amax_carry);
+                }
             }
 
             // ---- phase 4: O out of tensor memory.  A thread holds 16 columns of its row; writing them
@@ -734,7 +769,6 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     // int8 output: every accumulator requantised with the head's output multiplier by the rule
                     // of the logits, clamp((acc*Mo + 2^(sh-1)) >> sh, -128, 127), in 64 bits (a handful of
                     // values per thread and tile); the tile is staged as plain rows of D bytes
-                    const int32_t out_mult = a.requant_mult[8 * head + 5];
                     const int64_t round = (int64_t)1 << (a.out_requant_shift - 1);
                     uint32_t packed[kCols / 4];
 #pragma unroll
@@ -776,6 +810,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             }
             // leave the loop together (the flag was sampled once, before the barrier above)
             if (*(volatile int *)&leave_flag) break;
+            cur = nxt;
+            cc = nc;
         }
         if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // smem must outlive the reads
     }
