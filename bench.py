@@ -50,13 +50,13 @@ MODE_FLAGS = {"u8div": 0, "u8clb": 2, "u16div": 1, "u16clb": 3}
 # the middle of the rotating-buffer loop without a cache flush in front of them (so that the lines
 # evicted by a launch are counted like in the timed loop); see profiles/.  None: not captured for
 # the kernel as it stands.
-NCU_TRAFFIC_BYTES = {"config2": 135.7e6, "config3": 67.2e6, "config4": 400.4e6, "config5": 176.3e6}
+NCU_TRAFFIC_BYTES = {"config2": 135.7e6, "config3": 67.2e6, "config4": 400.4e6, "config5": 176.4e6}
 
 # Fused kernel: warp instructions on the integer (ALU) pipe per launch of workload 5, from the ncu
 # capture under profiles/ (sm__inst_executed_pipe_alu).  The pipe issues one warp instruction per
 # two cycles and scheduler (16 lanes per SM sub-partition), so its peak on 148 SMs x 4 schedulers at
 # 1.965 GHz is 148 * 4 * 1.965e9 / 2 warp instructions per second.
-FUSED_ALU_WARP_INSTR = {"config5": 59.9e6}
+FUSED_ALU_WARP_INSTR = {"config5": 59.7e6}
 ALU_PIPE_PEAK_WARP_INSTR_S = 148 * 4 * 1.965e9 / 2
 
 
