@@ -42,8 +42,7 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 }
 
 // Streaming accesses: nothing is read or written twice, so neither loads nor stores allocate in L1.
-// EVICT_FIRST also marks the loaded lines as the first to leave L2 (measured: 3 % faster for the
-// lane-per-row shapes, 5 % slower for 512-key rows, nothing in between: used for G = 1 only).
+// EVICT_FIRST also marks the loaded lines as the first to leave L2 (which shapes use it: see the kernel).
 template <bool EVICT_FIRST>
 __device__ __forceinline__ void ldg256(const void *p, uint32_t (&r)[8]) {
     if (EVICT_FIRST) {
@@ -115,6 +114,13 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     constexpr int RW = 32 / G;      // rows per warp
     constexpr int NW = CW * V;      // 32-bit words of logits per lane
     constexpr int CB = 4 * CW;      // bytes (keys) per chunk
+    // Two ways through L2, chosen by measurement (side by side, per shape).  A lane that holds a whole row of
+    // 96 and more keys, or 16-byte chunks, marks its loaded lines evict-first and prefetches nothing (2 to 5 %
+    // faster than the other way on 48, 96, 144 and 160 keys).  Every other shape -- lane groups, and a lane per
+    // row of 32 or 64 keys -- loads at normal priority behind one bulk prefetch per CTA (64 keys: 1.2 % faster
+    // than evict-first loads without a prefetch, 2 to 5 % in the leading-bit form and on longer launches;
+    // evict-first loads behind a prefetch are the worst combination).
+    constexpr bool kEvictFirst = G == 1 && (V > 2 || CW != 8);
     const int lane = threadIdx.x & 31;
     const int sub = lane % G;
     const uint32_t row = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * RW + lane / G;
@@ -131,10 +137,9 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
     // Before the wait: one bulk prefetch of the CTA's rows (they are contiguous) into L2.  A prefetch is safe
     // whatever the previous kernel of the stream still writes, because L2 is the point of coherence; in the first
     // wave it runs while that kernel drains, and in every wave the request leaves a prologue earlier than the
-    // lanes' own loads: 4 to 7 % on 128-key causal heads, 1 % on 512-key rows.  Not for the lane-per-row shapes:
-    // measured no gain or a loss there (their loads mark the lines evict-first, a prefetched line keeps its normal
-    // priority and crowds the output out of L2).
-    if (G > 1 && threadIdx.x == 0) {
+    // lanes' own loads: 4 to 7 % on 128-key causal heads, 1 % on 512-key rows.  Not for the evict-first shapes
+    // (a prefetched line keeps its normal priority and crowds the output out of L2).
+    if (!kEvictFirst && threadIdx.x == 0) {
         const uint32_t cta_row0 = blockIdx.x * (blockDim.x >> 5) * RW;        // (they are contiguous; row0 < rows)
         const uint32_t bytes = min((blockDim.x >> 5) * RW, (uint32_t)a.rows - cta_row0) * (uint32_t)a.Lk;   // a multiple of 16
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(x_all + (int64_t)cta_row0 * a.Lk), "r"(bytes));
@@ -164,8 +169,8 @@ __global__ void __launch_bounds__(256) rows_split_kernel(const int8_t *x_all, vo
         full[v] = !CAUSAL || __all_sync(0xffffffffu, cnt[v] == CB);
         uint32_t w[CW];
         if (cnt[v] > 0) {
-            if constexpr (CW == 8) ldg256<G == 1>(x_row + col, w);
-            else ldg128<G == 1>(x_row + col, w);
+            if constexpr (CW == 8) ldg256<kEvictFirst>(x_row + col, w);
+            else ldg128<kEvictFirst>(x_row + col, w);
         } else {
 #pragma unroll
             for (int k = 0; k < CW; ++k) w[k] = kMinus128x4;
