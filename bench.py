@@ -50,7 +50,7 @@ MODE_FLAGS = {"u8div": 0, "u8clb": 2, "u16div": 1, "u16clb": 3}
 # the middle of the rotating-buffer loop without a cache flush in front of them (so that the lines
 # evicted by a launch are counted like in the timed loop); see profiles/.  None: not captured for
 # the kernel as it stands.
-NCU_TRAFFIC_BYTES = {"config2": 135.7e6, "config3": 67.2e6, "config4": 400.4e6, "config5": 176.4e6}
+NCU_TRAFFIC_BYTES = {"config2": 135.1e6, "config3": 67.0e6, "config4": 400.0e6, "config5": 176.0e6}
 
 # Fused kernel: warp instructions on the integer (ALU) pipe per launch of workload 5, from the ncu
 # capture under profiles/ (sm__inst_executed_pipe_alu).  The pipe issues one warp instruction per
