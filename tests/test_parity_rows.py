@@ -120,6 +120,42 @@ def test_in_place(ctx, oracle, hccs):
             _check(ctx, oracle, wl, flags, inplace=True)
 
 
+@pytest.mark.parametrize("shape,flags", [((400, 4, 64, 64), 0), ((400, 4, 64, 64), 2), ((50, 8, 128, 128), 4),
+                                         ((2, 12, 512, 512), 0), ((800, 4, 64, 32), 0), ((3000, 4, 64, 64), 0)])
+def test_chain_of_dependent_launches(ctx, oracle, hccs, shape, flags):
+    """X -> A -> B -> C, three launches back to back on one stream with no synchronisation, each reading as
+    int8 logits the bytes the previous one wrote.  With programmatic dependent launch a kernel's prologue --
+    and its L2 prefetch of the input -- runs while the previous kernel still writes that input (the grids
+    here are mostly smaller than one wave, so that both kernels are resident together); A, B and C hold
+    other bytes beforehand, so a load that did not wait for the previous kernel shows."""
+    import torch
+    wl = hccs.workloads.make_rows(77, shape, kind="gauss")
+    ctx.hccs_params_upload(wl.theta, wl.n_design)
+    mode = oracle_mode(oracle, flags)
+    want, stages = wl.logits, []
+    for _ in range(3):
+        want = oracle.forward(want.view(np.int8), wl.theta, mode, threads=16).view(np.int8)
+        stages.append(want)
+    dev = torch.device("cuda", ctx.device)
+    x = torch.from_numpy(wl.logits).to(dev)
+    bufs = [torch.empty(shape, dtype=torch.int8, device=dev) for _ in range(3)]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234)
+    for rep in range(12):
+        for t in bufs:
+            t.view(torch.uint8).copy_(torch.randint(0, 256, shape, dtype=torch.uint8, device=dev, generator=gen))
+        torch.cuda.synchronize()
+        src = x
+        for t in bufs:
+            ctx.hccs_forward(src, t.view(torch.uint8), flags)
+            src = t
+        torch.cuda.synchronize()
+        for k, t in enumerate(bufs):
+            assert_same(t.cpu().numpy().view(np.uint8), stages[k].view(np.uint8),
+                        f"chain stage {k + 1} shape={shape} flags={flags} repeat={rep}")
+    assert ctx.hccs_device_status() == 0
+
+
 def test_many_heads_and_odd_head_count(ctx, oracle, hccs):
     wl = hccs.workloads.make_rows(5, (3, 67, 3, 64), kind="gauss")
     _check(ctx, oracle, wl, 0)
